@@ -1,0 +1,213 @@
+/*
+ * liblightkv -- prefill-time vision-token compression (LightKV) for one B200.
+ *
+ * C ABI.  Every pointer below is marked HOST or DEVICE.  The caller owns all
+ * device buffers and the stream; the library allocates no device memory, never
+ * synchronises, never changes the current device and enqueues only on the
+ * stream it is given.  A plan owns host memory only and is immutable after
+ * creation; concurrent calls that use distinct workspaces are allowed.
+ *
+ * Every function returns an int status (LIGHTKV_OK = 0, negative = error).
+ * Conditions that the host can see (shapes, modes, capacities, alignment) are
+ * returned before anything is launched.  Conditions only visible on the device
+ * (positions not ascending, a vanishing weight sum, a bounded wait that ran
+ * out) set bits in the optional DEVICE status word and leave the outputs
+ * defined; kernels always run to completion.
+ *
+ * Method (section "LightKV" of the paper): at a scheduled decoder layer the
+ * vision tokens are put back on their image grid, cut into w x w windows
+ * ("Window partitioning"), split alternately into sets A and B inside every
+ * window (Step 1), scored with the feature divergence FD = 1 - cosine
+ * (Eq. "similarity", Step 2), the lowest-FD A nodes are attached to their best
+ * B node, and every B node becomes the xi-weighted mean of itself and the A
+ * nodes attached to it (Eq. "message-passing", Step 3), where xi_i is the
+ * attention mass vision token i puts on the prompt tokens, summed over heads
+ * (Eq. "attention-factor").  Merged A nodes are dropped (Step 4) and the
+ * survivors are emitted in their original order (Step 5).  The same map is
+ * applied to the layer's K/V cache ("key and value tokens are compressed
+ * simultaneously", appendix "Method overview").
+ */
+#ifndef LIGHTKV_H_
+#define LIGHTKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LIGHTKV_VERSION 100
+
+/* status codes */
+#define LIGHTKV_OK               0
+#define LIGHTKV_ERR_INVALID_ARG (-1)
+#define LIGHTKV_ERR_UNSUPPORTED (-2)
+#define LIGHTKV_ERR_WORKSPACE   (-3)
+#define LIGHTKV_ERR_CAPACITY    (-4)
+#define LIGHTKV_ERR_CUDA        (-5)
+#define LIGHTKV_ERR_TIMEOUT     (-6)
+
+/* bits of the DEVICE status word */
+#define LIGHTKV_STATUS_POS_ORDER   1u   /* positions not strictly ascending / out of the grid */
+#define LIGHTKV_STATUS_ZERO_WEIGHT 2u   /* a group's xi sum vanished: plain mean was used      */
+#define LIGHTKV_STATUS_TIMEOUT     4u   /* a bounded device-side wait expired                  */
+#define LIGHTKV_STATUS_COUNT       8u   /* n_vis[b] exceeds the stage's capacity               */
+
+/* storage / arithmetic type of hidden states, Q, K, V */
+#define LIGHTKV_BF16 0   /* bf16 storage, fp32 accumulation                     */
+#define LIGHTKV_FP32 1   /* fp32 storage and arithmetic (SIMT kernels only)     */
+
+/* where xi comes from */
+#define LIGHTKV_XI_GIVEN     0   /* caller passes xi                                                  */
+#define LIGHTKV_XI_ATTN_FULL 1   /* computed from Q and K: causal softmax rows, Eq. "attention-factor" */
+#define LIGHTKV_XI_ATTN_LSE  2   /* as ATTN_FULL, but the row log-sum-exp comes from the caller's
+                                    fused attention, so only the prompt keys are visited              */
+#define LIGHTKV_XI_UNIFORM   3   /* xi = 1 (plain group mean; the paper's "uniform" ablation)          */
+
+/* K/V operator */
+#define LIGHTKV_KV_MERGE  0      /* K'_o = sum over the group of weight_i K_i (same weights as hidden) */
+#define LIGHTKV_KV_GATHER 1      /* K'_o = row of the group's surviving token                          */
+
+/* contraction engine */
+#define LIGHTKV_ENGINE_AUTO 0    /* tcgen05 tensor-core kernels for bf16 where the shape allows */
+#define LIGHTKV_ENGINE_SIMT 1    /* fp32 FMA kernels                                            */
+
+typedef struct lightkv_plan lightkv_plan_t;
+
+typedef struct { int32_t rows, cols; } lightkv_tile_t;   /* grid of one image tile / video frame */
+
+/* Model shape and schedule (Lambda, W, P of section "Hierarchical structure").
+ * All pointers HOST; copied by lightkv_plan. */
+typedef struct {
+  uint32_t struct_size;            /* sizeof(lightkv_config_t) */
+  int32_t  batch;                  /* samples per call */
+  int32_t  hidden;                 /* d; multiple of 8 */
+  int32_t  n_q_heads, n_kv_heads;  /* H, H_kv; H % H_kv == 0 */
+  int32_t  head_dim;               /* multiple of 8; tensor-core xi needs 64 or 128 */
+  int32_t  n_layers;               /* L, used by the accounting only */
+  int32_t  n_tiles;                /* >= 1; sum of rows*cols = vision tokens before stage 0 */
+  const lightkv_tile_t* tiles;
+  int32_t  n_stages;               /* s */
+  const int32_t* layers;           /* lambda_i, ascending, in [1, L] */
+  const int32_t* windows;          /* w_i: windows per axis, applied to every tile separately */
+  const double*  keep;             /* 1 - rho_i, each in [0.5, 1] */
+  int32_t  max_text;               /* upper bound on text rows (before + after the vision block) */
+  int32_t  dtype;                  /* LIGHTKV_BF16 | LIGHTKV_FP32 */
+  int32_t  xi_mode;                /* LIGHTKV_XI_* */
+  int32_t  engine;                 /* LIGHTKV_ENGINE_* */
+} lightkv_config_t;
+
+typedef struct {
+  int32_t layer;                   /* lambda_i */
+  int32_t window;                  /* w_i */
+  double  keep;                    /* 1 - rho_i */
+  int32_t cap_in;                  /* upper bound on vision tokens per sample entering the stage;
+                                      also the row stride of every per-token int/float array      */
+  int32_t cap_out;                 /* same, leaving it (= cap_in of the next stage)               */
+  int32_t n_windows;               /* windows per sample */
+  int32_t counts_exact;            /* 1: every sample holds exactly cap_in / cap_out tokens when
+                                      it entered stage 0 with the full grid (host simulation)     */
+  int32_t uses_tensor_cores;       /* 1: the FD and xi contractions of this stage run on tcgen05  */
+  size_t  workspace_bytes;         /* DEVICE scratch lightkv_compress_layer needs                 */
+} lightkv_stage_info_t;
+
+/* Build a plan.  HOST only, no CUDA call.  *out receives the plan.
+ * Errors: INVALID_ARG (NULL, non-positive sizes, keep outside [0.5,1], w larger than a tile side,
+ * layers not ascending), UNSUPPORTED (more windows per sample or more tiles than the kernels take). */
+int  lightkv_plan(const lightkv_config_t* config, lightkv_plan_t** out);
+int  lightkv_plan_stage_info(const lightkv_plan_t* plan, int32_t stage, lightkv_stage_info_t* info);
+void lightkv_plan_destroy(lightkv_plan_t* plan);
+
+/* Eq. "complexity": fraction of the v * L vision tokens still processed under the plan's schedule
+ * (rho_i taken from the plan).  Returns a negative value on a NULL plan. */
+double lightkv_plan_retention(const lightkv_plan_t* plan);
+
+/* One compression stage on a batch (Steps 1-5).  Sample b's sequence is
+ *   [ vis_begin text rows | n_vis[b] vision rows | n_text_after rows ]
+ * inside a buffer whose rows are `row_stride` elements apart.  All strides are
+ * in ELEMENTS; the last dimension (hidden or head_dim) is contiguous; every row
+ * must start on a 16-byte boundary. */
+typedef struct {
+  uint32_t struct_size;            /* sizeof(lightkv_layer_args_t) */
+  int32_t  stage;
+  int32_t  vis_begin;              /* text rows before the vision block */
+  int32_t  n_text_after;           /* rows after it (copied through) */
+  int32_t  text_begin, text_end;   /* prompt-token set J = [text_begin, text_end) within [0, vis_begin] */
+
+  const void* hidden;              /* DEVICE [B, N, d] */
+  int64_t hidden_batch_stride, hidden_row_stride;
+  void*   hidden_out;              /* DEVICE [B, N', d]; must not overlap hidden */
+  int64_t hidden_out_batch_stride, hidden_out_row_stride;
+
+  const void* q;                   /* DEVICE [B, H, N, dh]   (ATTN_FULL, ATTN_LSE) */
+  int64_t q_batch_stride, q_head_stride, q_row_stride;
+  const void* k;                   /* DEVICE [B, H_kv, N, dh] (ATTN_FULL, ATTN_LSE) */
+  int64_t k_batch_stride, k_head_stride, k_row_stride;
+  const float* lse;                /* DEVICE [B, H, N] natural-log row log-sum-exp of the scaled
+                                      causal logits (ATTN_LSE) */
+  int64_t lse_batch_stride, lse_head_stride;
+  const float* xi;                 /* DEVICE [B, cap_in] (GIVEN) */
+
+  const int32_t* n_vis;            /* DEVICE [B]; NULL = cap_in for every sample */
+  const int32_t* pos;              /* DEVICE [B, cap_in] original flat grid positions, strictly
+                                      ascending per sample; NULL = 0..n-1 (stage 0, full grid) */
+
+  int32_t* n_vis_out;              /* DEVICE [B] */
+  int32_t* pos_out;                /* DEVICE [B, cap_out] */
+  /* the merge map of the stage */
+  int32_t* dst;                    /* DEVICE [B, cap_in]   output slot of every input vision token */
+  float*   weight;                 /* DEVICE [B, cap_in]   its weight xi_i / (group sum) */
+  int32_t* grp_off;                /* DEVICE [B, cap_out+1] slot o gathers grp_src[grp_off[o] .. grp_off[o+1]) */
+  int32_t* grp_src;                /* DEVICE [B, cap_in]   member token indices, survivor first */
+  float*   xi_out;                 /* DEVICE [B, cap_in] the xi that was used; may be NULL */
+
+  uint32_t* status;                /* DEVICE, one word, OR-ed into; may be NULL */
+  void*   workspace;               /* DEVICE, 256-byte aligned */
+  size_t  workspace_bytes;
+  void*   stream;                  /* cudaStream_t */
+} lightkv_layer_args_t;
+
+/* Enqueue window build, xi, FD + best partner, selection + merge map and the
+ * weighted merge of the hidden states.  Errors: INVALID_ARG, WORKSPACE (too
+ * small), UNSUPPORTED (mode / dtype / engine combination), CUDA (launch failed). */
+int lightkv_compress_layer(const lightkv_plan_t* plan, const lightkv_layer_args_t* args);
+
+/* Apply a stage's merge map to one layer's K and V (out of place).
+ * Contiguous: element (b, h, n, :) of a tensor lives at
+ *   base + b*batch_stride + h*head_stride + n*row_stride.
+ * Paged (page_size > 0): token n of sample b lives in page block_table[b*max_blocks + n/page_size] at
+ *   base + page*page_stride + h*head_stride + (n % page_size)*row_stride.
+ * Text rows are copied; vision rows are merged or gathered per `mode`. */
+typedef struct {
+  uint32_t struct_size;            /* sizeof(lightkv_kv_args_t) */
+  int32_t  stage;
+  int32_t  vis_begin, n_text_after;
+  int32_t  mode;                   /* LIGHTKV_KV_* */
+  const int32_t* n_vis;            /* DEVICE [B] or NULL (= cap_in) */
+  const int32_t* n_vis_out;        /* DEVICE [B] */
+  const int32_t* grp_off;          /* DEVICE, from lightkv_compress_layer */
+  const int32_t* grp_src;
+  const float*   weight;
+  const void* k_src; const void* v_src;      /* DEVICE */
+  void* k_dst; void* v_dst;                  /* DEVICE; must not overlap the sources */
+  int64_t src_batch_stride, src_head_stride, src_row_stride;
+  int64_t dst_batch_stride, dst_head_stride, dst_row_stride;
+  int32_t page_size;               /* 0 = contiguous */
+  int32_t max_blocks;              /* row stride of the block tables */
+  const int32_t* src_block_table;  /* DEVICE [B, max_blocks] */
+  const int32_t* dst_block_table;  /* DEVICE [B, max_blocks] */
+  int64_t src_page_stride, dst_page_stride;
+  uint32_t* status;                /* DEVICE, may be NULL */
+  void* stream;
+} lightkv_kv_args_t;
+
+int lightkv_compact_kv(const lightkv_plan_t* plan, const lightkv_kv_args_t* args);
+
+const char* lightkv_status_string(int status);
+int lightkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* LIGHTKV_H_ */

@@ -1,0 +1,41 @@
+// Host-side launch interface between the C ABI (lightkv_api.cu) and the kernel files.
+#pragma once
+#include "common.cuh"
+
+namespace lkv {
+
+struct LayerLaunch {
+  int batch, hidden, n_q_heads, n_kv_heads, head_dim;
+  int dtype, xi_mode;
+  double keep;
+  Geometry geo;
+  Workspace ws;
+  const lightkv_layer_args_t* a;
+  cudaStream_t stream;
+};
+
+// window build (Step 1 and "Window partitioning")
+cudaError_t launch_window_build(const LayerLaunch& L);
+// FD + best partner per A node (Step 2), fp32 FMA path
+cudaError_t launch_fd_simt(const LayerLaunch& L);
+// xi per head (Eq. "attention-factor"), fp32 FMA path; handles ATTN_FULL and ATTN_LSE
+cudaError_t launch_xi_simt(const LayerLaunch& L);
+// head sum of xi, ranking, merge map, weights (Steps 2-5)
+cudaError_t launch_select_map(const LayerLaunch& L);
+// weighted merge of the hidden states (Eq. "message-passing")
+cudaError_t launch_merge_rows(const LayerLaunch& L);
+
+struct KvLaunch {
+  int batch, n_kv_heads, head_dim, dtype, cap_in, cap_out;
+  const lightkv_kv_args_t* a;
+  cudaStream_t stream;
+};
+cudaError_t launch_kv_compact(const KvLaunch& K);
+
+// tcgen05 paths (lightkv_tc.cu).  `supported` queries are host-only.
+bool tc_fd_supported(int hidden);
+bool tc_xi_supported(int head_dim);
+cudaError_t launch_fd_tc(const LayerLaunch& L);
+cudaError_t launch_xi_tc(const LayerLaunch& L);
+
+}  // namespace lkv

@@ -1,0 +1,795 @@
+// liblightkv kernels, part 1: window build, fp32-FMA contractions (FD, xi), selection + merge map,
+// weighted merge of hidden states, K/V merge-compaction.  sm_100a.
+#include "launch.h"
+
+namespace lkv {
+
+__device__ inline void set_status(uint32_t* status, uint32_t bit) {
+  if (status) atomicOr(status, bit);
+}
+
+// =====================================================================================================
+// Window build ("Window partitioning", Step 1).  One CTA per sample.
+// Every token gets its window id from its original grid position; tokens of a window are ranked in
+// storage order (positions ascend with storage, so this is position order).  Rank l even -> set A
+// (the paper's 1st, 3rd, ... token), odd -> set B.  A and B nodes are listed window by window.
+// Stable ranking without sorting: each warp owns a contiguous segment of the tokens and a private row
+// of per-window counters; an exclusive prefix over the 32 rows gives every warp its starting rank.
+// =====================================================================================================
+__global__ void __launch_bounds__(1024)
+window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __restrict__ n_vis,
+                    Workspace ws, uint32_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int nW = g.n_windows;
+  uint16_t* cnt = reinterpret_cast<uint16_t*>(smem_raw);                        // [32][nW]
+  int* wsum = reinterpret_cast<int*>(smem_raw + ((size_t(32) * nW * 2 + 15) & ~size_t(15)));  // [nW+1]
+  int* asum = wsum + nW + 1;                                                    // [nW+1]
+
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+  int n = n_vis ? n_vis[b] : ws.cap_in;
+  if (n > ws.cap_in) { n = ws.cap_in; if (tid == 0) set_status(status, LIGHTKV_STATUS_COUNT); }
+  if (n < 0) n = 0;
+  const int* pos = pos_all ? pos_all + size_t(b) * ws.cap_in : nullptr;
+  int* tok_win = ws.tok_win + size_t(b) * ws.cap_in;
+  int* tok_l = ws.tok_l + size_t(b) * ws.cap_in;
+  int* a_tok = ws.a_tok + size_t(b) * ws.cap_a;
+  int* a_win = ws.a_win + size_t(b) * ws.cap_a;
+  int* b_tok = ws.b_tok + size_t(b) * ws.cap_b;
+
+  for (int i = tid; i < 32 * nW; i += blockDim.x) cnt[i] = 0;
+  __syncthreads();
+
+  const int seg = (n + 31) / 32;
+  const int s0 = min(n, wp * seg), s1 = min(n, s0 + seg);
+
+  // pass A: window id of every token, per-warp per-window counts
+  for (int base = s0; base < s1; base += 32) {
+    const int i = base + lane;
+    const bool act = i < s1;
+    const unsigned amask = __ballot_sync(0xffffffffu, act);
+    if (act) {
+      const int p = pos ? pos[i] : i;
+      int w = window_of(g, p);
+      const int prev = (i > 0) ? (pos ? pos[i - 1] : i - 1) : -1;
+      if (w < 0 || p <= prev) { set_status(status, LIGHTKV_STATUS_POS_ORDER); if (w < 0) w = 0; }
+      tok_win[i] = w;
+      const unsigned peers = __match_any_sync(amask, w);
+      if (lane == __ffs(peers) - 1) cnt[wp * nW + w] += (uint16_t)__popc(peers);
+    }
+    __syncwarp();
+  }
+  __syncthreads();
+
+  // exclusive prefix over the 32 warp rows, window totals
+  for (int w = tid; w < nW; w += blockDim.x) {
+    int run = 0;
+    for (int k = 0; k < 32; ++k) {
+      const int c = cnt[k * nW + w];
+      cnt[k * nW + w] = (uint16_t)run;
+      run += c;
+    }
+    wsum[w] = run;
+  }
+  __syncthreads();
+
+  // exclusive scans over windows: token offsets (wsum) and A-entry offsets (asum)
+  if (wp == 0) {
+    const int chunk = (nW + 31) / 32;
+    const int lo = min(nW, lane * chunk), hi = min(nW, lo + chunk);
+    int s = 0, sa = 0;
+    for (int w = lo; w < hi; ++w) { s += wsum[w]; sa += (wsum[w] + 1) >> 1; }
+    int xs = s, xa = sa;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, xs, o), ta = __shfl_up_sync(0xffffffffu, xa, o);
+      if (lane >= o) { xs += t; xa += ta; }
+    }
+    xs -= s; xa -= sa;
+    for (int w = lo; w < hi; ++w) {
+      const int c = wsum[w];
+      wsum[w] = xs; asum[w] = xa;
+      xs += c; xa += (c + 1) >> 1;
+    }
+    if (lane == 31) { wsum[nW] = xs; asum[nW] = xa; }
+  }
+  __syncthreads();
+  for (int w = tid; w <= nW; w += blockDim.x) {
+    ws.win_off[size_t(b) * (nW + 1) + w] = wsum[w];
+    ws.a_off[size_t(b) * (nW + 1) + w] = asum[w];
+  }
+
+  // pass B: local rank, A / B entry lists
+  for (int base = s0; base < s1; base += 32) {
+    const int i = base + lane;
+    const bool act = i < s1;
+    const unsigned amask = __ballot_sync(0xffffffffu, act);
+    if (act) {
+      const int w = tok_win[i];
+      const unsigned peers = __match_any_sync(amask, w);
+      const int before = cnt[wp * nW + w];
+      __syncwarp(amask);
+      if (lane == __ffs(peers) - 1) cnt[wp * nW + w] = (uint16_t)(before + __popc(peers));
+      __syncwarp(amask);
+      const int l = before + __popc(peers & ((1u << lane) - 1u));
+      tok_l[i] = l;
+      if (l & 1) {
+        const int e = (wsum[w] - asum[w]) + (l >> 1);
+        if (e < ws.cap_b) b_tok[e] = i;
+      } else {
+        const int e = asum[w] + (l >> 1);
+        if (e < ws.cap_a) { a_tok[e] = i; a_win[e] = w; }
+      }
+    }
+    __syncwarp();
+  }
+}
+
+cudaError_t launch_window_build(const LayerLaunch& L) {
+  const int nW = L.geo.n_windows;
+  const size_t smem = ((size_t(32) * nW * 2 + 15) & ~size_t(15)) + size_t(2) * (nW + 1) * sizeof(int);
+  cudaError_t e = cudaFuncSetAttribute(window_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       200 * 1024);
+  if (e != cudaSuccess) return e;
+  window_build_kernel<<<L.batch, 1024, smem, L.stream>>>(L.geo, L.a->pos, L.a->n_vis, L.ws, L.a->status);
+  return cudaGetLastError();
+}
+
+// =====================================================================================================
+// FD + best partner, fp32 FMA path (Eq. "similarity", Step 2).
+// One CTA per (sample, tile of 32 A entries).  The B entries of the windows the tile touches are
+// visited in chunks of 64; G = X_A X_B^T accumulates in registers over k-chunks of 32 staged in smem,
+// squared norms accumulate from the same staged tiles.  Every A row then scans the FD of its own
+// window's B entries in ascending order (strict <, so ties go to the lowest B index).
+// =====================================================================================================
+constexpr int FD_TA = 32, FD_TB = 64, FD_KC = 32;
+
+template <typename T>
+__device__ inline void load4(const T* p, float (&f)[4]);
+template <>
+__device__ inline void load4<float>(const float* p, float (&f)[4]) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+template <>
+__device__ inline void load4<__nv_bfloat16>(const __nv_bfloat16* p, float (&f)[4]) {
+  const uint2 v = *reinterpret_cast<const uint2*>(p);
+  f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+  f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_stride, int vis_begin,
+               int d, Workspace ws) {
+  __shared__ float As[FD_TA][FD_KC + 1];
+  __shared__ float Bs[FD_TB][FD_KC + 1];
+  __shared__ float Gs[FD_TA][FD_TB + 1];
+  __shared__ float a_ss[FD_TA], b_ss[FD_TB];
+  __shared__ int a_row[FD_TA], b_row[FD_TB], a_lo[FD_TA], a_hi[FD_TA];
+
+  const int b = blockIdx.y, tid = threadIdx.x;
+  const int nW = ws.n_windows;
+  const int* win_off = ws.win_off + size_t(b) * (nW + 1);
+  const int* a_off = ws.a_off + size_t(b) * (nW + 1);
+  const int* a_tok = ws.a_tok + size_t(b) * ws.cap_a;
+  const int* a_win = ws.a_win + size_t(b) * ws.cap_a;
+  const int* b_tok = ws.b_tok + size_t(b) * ws.cap_b;
+  const int n_a = a_off[nW];
+  const int e0 = blockIdx.x * FD_TA;
+  if (e0 >= n_a) return;
+  const int ne = min(FD_TA, n_a - e0);
+  const T* x = hidden + size_t(b) * batch_stride + size_t(vis_begin) * row_stride;
+
+  if (tid < FD_TA) {
+    if (tid < ne) {
+      const int w = a_win[e0 + tid];
+      a_row[tid] = a_tok[e0 + tid];
+      a_lo[tid] = win_off[w] - a_off[w];
+      a_hi[tid] = win_off[w + 1] - a_off[w + 1];
+    } else {
+      a_row[tid] = -1; a_lo[tid] = 0; a_hi[tid] = 0;
+    }
+  }
+  __syncthreads();
+  const int bb0 = a_lo[0], bb1 = a_hi[ne - 1];
+
+  const int tx = tid & 15, ty = tid >> 4;            // 4 B columns x 2 A rows per thread
+  float best_f = 3.0e38f;                            // threads < ne: running minimum of their A row
+  int best_tok = -1;
+  float ssa = 0.f;                                   // threads < FD_TA: squared norm of A row tid
+
+  for (int cb = bb0; cb < bb1; cb += FD_TB) {
+    const int nb = min(FD_TB, bb1 - cb);
+    if (tid < FD_TB) b_row[tid] = tid < nb ? b_tok[cb + tid] : -1;
+    float acc[2][4] = {};
+    float ssb = 0.f;                                 // threads 32..95: squared norm of B row tid-32
+    const bool first = (cb == bb0);
+    __syncthreads();
+    for (int k0 = 0; k0 < d; k0 += FD_KC) {
+      {  // stage A tile: 32 x 32, 4 elements per thread
+        const int r = tid >> 3, c = (tid & 7) * 4;
+        float f[4] = {0.f, 0.f, 0.f, 0.f};
+        if (a_row[r] >= 0 && k0 + c < d) load4<T>(x + size_t(a_row[r]) * row_stride + k0 + c, f);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) As[r][c + j] = f[j];
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {  // stage B tile: 64 x 32
+        const int r = (tid >> 3) + half * 32, c = (tid & 7) * 4;
+        float f[4] = {0.f, 0.f, 0.f, 0.f};
+        if (b_row[r] >= 0 && k0 + c < d) load4<T>(x + size_t(b_row[r]) * row_stride + k0 + c, f);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) Bs[r][c + j] = f[j];
+      }
+      __syncthreads();
+#pragma unroll 8
+      for (int kk = 0; kk < FD_KC; ++kk) {
+        const float a0 = As[2 * ty][kk], a1 = As[2 * ty + 1][kk];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float bv = Bs[4 * tx + j][kk];
+          acc[0][j] = fmaf(a0, bv, acc[0][j]);
+          acc[1][j] = fmaf(a1, bv, acc[1][j]);
+        }
+      }
+      if (first && tid < FD_TA) {
+        for (int kk = 0; kk < FD_KC; ++kk) ssa = fmaf(As[tid][kk], As[tid][kk], ssa);
+      } else if (tid >= 32 && tid < 32 + FD_TB) {
+        for (int kk = 0; kk < FD_KC; ++kk) ssb = fmaf(Bs[tid - 32][kk], Bs[tid - 32][kk], ssb);
+      }
+      __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) Gs[2 * ty + i][4 * tx + j] = acc[i][j];
+    if (first && tid < FD_TA) a_ss[tid] = ssa;
+    if (tid >= 32 && tid < 32 + FD_TB) b_ss[tid - 32] = ssb;
+    __syncthreads();
+    if (tid < ne) {
+      const int lo = max(a_lo[tid], cb), hi = min(a_hi[tid], cb + nb);
+      const float na = sqrtf(a_ss[tid]);
+      for (int e = lo; e < hi; ++e) {
+        const float den = na * sqrtf(b_ss[e - cb]);
+        const float cosv = den > 0.f ? Gs[tid][e - cb] / den : 0.f;
+        const float fd = 1.0f - cosv;
+        if (fd < best_f) { best_f = fd; best_tok = b_row[e - cb]; }
+      }
+    }
+    __syncthreads();
+  }
+  if (tid < ne) {
+    ws.a_f[size_t(b) * ws.cap_a + e0 + tid] = best_f;
+    ws.a_best[size_t(b) * ws.cap_a + e0 + tid] = best_tok;
+  }
+}
+
+cudaError_t launch_fd_simt(const LayerLaunch& L) {
+  const dim3 grid((L.ws.cap_a + FD_TA - 1) / FD_TA, L.batch);
+  if (L.dtype == LIGHTKV_BF16)
+    fd_simt_kernel<__nv_bfloat16><<<grid, 256, 0, L.stream>>>(
+        static_cast<const __nv_bfloat16*>(L.a->hidden), L.a->hidden_batch_stride, L.a->hidden_row_stride,
+        L.a->vis_begin, L.hidden, L.ws);
+  else
+    fd_simt_kernel<float><<<grid, 256, 0, L.stream>>>(
+        static_cast<const float*>(L.a->hidden), L.a->hidden_batch_stride, L.a->hidden_row_stride,
+        L.a->vis_begin, L.hidden, L.ws);
+  return cudaGetLastError();
+}
+
+// =====================================================================================================
+// xi per head, fp32 FMA path (Eq. "attention-factor" with the causal softmax rows of Eq.
+// "attention-matrix").  One CTA per (tile of 32 vision queries, head, sample).  Keys 0..s_i are visited
+// in tiles of 64 with an online (running-maximum) softmax that carries two sums per row: all visible
+// keys and the prompt keys J.  Output per head: sum_J / sum_all.  With a caller-supplied row
+// log-sum-exp only the prompt keys are visited: sum_J exp(logit - lse).
+// =====================================================================================================
+constexpr int XI_TQ = 32, XI_TK = 64;
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+xi_simt_kernel(const T* __restrict__ q, int64_t q_bs, int64_t q_hs, int64_t q_rs,
+               const T* __restrict__ k, int64_t k_bs, int64_t k_hs, int64_t k_rs,
+               const float* __restrict__ lse, int64_t lse_bs, int64_t lse_hs,
+               const int* __restrict__ n_vis, int vis_begin, int text_begin, int text_end,
+               int n_q_heads, int n_kv_heads, int dh, Workspace ws) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int ld = dh + 1;
+  float* Qs = reinterpret_cast<float*>(smem_raw);       // [XI_TQ][ld]
+  float* Ks = Qs + XI_TQ * ld;                          // [XI_TK][ld]
+  float* Ss = Ks + XI_TK * ld;                          // [XI_TQ][XI_TK + 1]
+
+  const int b = blockIdx.z, h = blockIdx.y, t0 = blockIdx.x * XI_TQ, tid = threadIdx.x;
+  int n = n_vis ? min(n_vis[b], ws.cap_in) : ws.cap_in;
+  if (t0 >= n) return;
+  const int nq = min(XI_TQ, n - t0);
+  const int hk = h / (n_q_heads / n_kv_heads);
+  const T* qh = q + size_t(b) * q_bs + size_t(h) * q_hs;
+  const T* kh = k + size_t(b) * k_bs + size_t(hk) * k_hs;
+  const float scale2 = 1.4426950408889634f / sqrtf((float)dh);      // logits in log2 units
+
+  for (int idx = tid; idx < XI_TQ * (dh / 4); idx += blockDim.x) {
+    const int r = idx / (dh / 4), c = (idx % (dh / 4)) * 4;
+    float f[4] = {0.f, 0.f, 0.f, 0.f};
+    if (r < nq) load4<T>(qh + size_t(vis_begin + t0 + r) * q_rs + c, f);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) Qs[r * ld + c + j] = f[j];
+  }
+
+  const int tx = tid & 15, ty = tid >> 4;
+  const int lane = tid & 31, wp = tid >> 5;             // softmax: warp wp owns rows 4*wp .. 4*wp+3
+  float m_run[4], l_all[4], l_txt[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { m_run[i] = -INFINITY; l_all[i] = 0.f; l_txt[i] = 0.f; }
+
+  const int s_last = vis_begin + t0 + nq - 1;           // last key any row of the tile may see
+  const int key_lo = lse ? text_begin : 0;
+  const int key_hi = lse ? min(text_end, s_last + 1) : s_last + 1;
+
+  for (int j0 = key_lo; j0 < key_hi; j0 += XI_TK) {
+    const int nk = min(XI_TK, key_hi - j0);
+    __syncthreads();
+    for (int idx = tid; idx < XI_TK * (dh / 4); idx += blockDim.x) {
+      const int r = idx / (dh / 4), c = (idx % (dh / 4)) * 4;
+      float f[4] = {0.f, 0.f, 0.f, 0.f};
+      if (r < nk) load4<T>(kh + size_t(j0 + r) * k_rs + c, f);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) Ks[r * ld + c + j] = f[j];
+    }
+    __syncthreads();
+    float acc[2][4] = {};
+    for (int kk = 0; kk < dh; ++kk) {
+      const float a0 = Qs[(2 * ty) * ld + kk], a1 = Qs[(2 * ty + 1) * ld + kk];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float bv = Ks[(4 * tx + j) * ld + kk];
+        acc[0][j] = fmaf(a0, bv, acc[0][j]);
+        acc[1][j] = fmaf(a1, bv, acc[1][j]);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) Ss[(2 * ty + i) * (XI_TK + 1) + 4 * tx + j] = acc[i][j] * scale2;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = 4 * wp + i;
+      if (r >= nq) continue;                            // warp-uniform
+      const int s_i = vis_begin + t0 + r;
+      float v[2];
+      bool ok[2], txt[2];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int j = j0 + lane + 32 * c;
+        ok[c] = (lane + 32 * c < nk) && j <= s_i;
+        txt[c] = ok[c] && j >= text_begin && j < text_end;
+        v[c] = ok[c] ? Ss[r * (XI_TK + 1) + lane + 32 * c] : -INFINITY;
+      }
+      if (lse) {
+        const float l2 = lse[size_t(b) * lse_bs + size_t(h) * lse_hs + s_i] * 1.4426950408889634f;
+        float p = (txt[0] ? exp2f(v[0] - l2) : 0.f) + (txt[1] ? exp2f(v[1] - l2) : 0.f);
+        for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
+        l_txt[i] += p;
+        continue;
+      }
+      float mx = fmaxf(v[0], v[1]);
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float m_new = fmaxf(m_run[i], mx);          // finite: key 0 is visible to every query
+      const float p0 = ok[0] ? exp2f(v[0] - m_new) : 0.f, p1 = ok[1] ? exp2f(v[1] - m_new) : 0.f;
+      float sa = p0 + p1, st = (txt[0] ? p0 : 0.f) + (txt[1] ? p1 : 0.f);
+      for (int o = 16; o > 0; o >>= 1) {
+        sa += __shfl_xor_sync(0xffffffffu, sa, o);
+        st += __shfl_xor_sync(0xffffffffu, st, o);
+      }
+      const float resc = exp2f(m_run[i] - m_new);       // 0 on the first tile (m_run = -inf)
+      l_all[i] = l_all[i] * resc + sa;
+      l_txt[i] = l_txt[i] * resc + st;
+      m_run[i] = m_new;
+    }
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = 4 * wp + i;
+      if (r < nq)
+        ws.xi_h[(size_t(b) * n_q_heads + h) * ws.cap_in + t0 + r] = lse ? l_txt[i] : l_txt[i] / l_all[i];
+    }
+  }
+}
+
+cudaError_t launch_xi_simt(const LayerLaunch& L) {
+  const lightkv_layer_args_t* a = L.a;
+  const int dh = L.head_dim;
+  const size_t smem = (size_t(XI_TQ + XI_TK) * (dh + 1) + size_t(XI_TQ) * (XI_TK + 1)) * sizeof(float);
+  const dim3 grid((L.ws.cap_in + XI_TQ - 1) / XI_TQ, L.n_q_heads, L.batch);
+  const float* lse = L.xi_mode == LIGHTKV_XI_ATTN_LSE ? a->lse : nullptr;
+  cudaError_t e;
+  if (L.dtype == LIGHTKV_BF16) {
+    auto kern = xi_simt_kernel<__nv_bfloat16>;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024)) != cudaSuccess)
+      return e;
+    kern<<<grid, 256, smem, L.stream>>>(
+        static_cast<const __nv_bfloat16*>(a->q), a->q_batch_stride, a->q_head_stride, a->q_row_stride,
+        static_cast<const __nv_bfloat16*>(a->k), a->k_batch_stride, a->k_head_stride, a->k_row_stride,
+        lse, a->lse_batch_stride, a->lse_head_stride, a->n_vis, a->vis_begin, a->text_begin, a->text_end,
+        L.n_q_heads, L.n_kv_heads, dh, L.ws);
+  } else {
+    auto kern = xi_simt_kernel<float>;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024)) != cudaSuccess)
+      return e;
+    kern<<<grid, 256, smem, L.stream>>>(
+        static_cast<const float*>(a->q), a->q_batch_stride, a->q_head_stride, a->q_row_stride,
+        static_cast<const float*>(a->k), a->k_batch_stride, a->k_head_stride, a->k_row_stride,
+        lse, a->lse_batch_stride, a->lse_head_stride, a->n_vis, a->vis_begin, a->text_begin, a->text_end,
+        L.n_q_heads, L.n_kv_heads, dh, L.ws);
+  }
+  return cudaGetLastError();
+}
+
+// =====================================================================================================
+// Selection + merge map (Steps 2-5).  One CTA per sample, phases separated by block barriers.
+//   0  xi = fixed-order sum over heads (or given / uniform)
+//   1  per window: r = removal_count(n_w); the r A entries with the smallest (FD, index) are selected
+//      (rank by counting; skipped when r = |A|); a selected A token records its best B token
+//   2  survivors (all B, unselected A) get consecutive output slots in storage (= position) order
+//   3  dst, pos_out
+//   4  group sizes -> grp_off (scan) ; 5 grp_src (survivor first, then its A members ascending) and
+//      weights xi_i / sum (summed in that fixed order)
+// =====================================================================================================
+struct SelectArgs {
+  int n_q_heads, xi_mode, cap_out;
+  double keep;
+  const int* n_vis;
+  const int* pos;
+  const float* xi_in;
+  int* n_vis_out;
+  int* pos_out;
+  int* dst;
+  float* weight;
+  int* grp_off;
+  int* grp_src;
+  float* xi_out;
+  uint32_t* status;
+};
+
+// exclusive scan of one value per thread across the CTA; returns the exclusive prefix, total in *total
+__device__ inline int block_exclusive_scan(int v, int* warp_sums /* [33] smem */, int* total) {
+  const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  int x = v;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += t;
+  }
+  __syncthreads();                       // warp_sums may still be read from the previous call
+  if (lane == 31) warp_sums[wp] = x;
+  __syncthreads();
+  if (wp == 0) {
+    int s = lane < nwarps ? warp_sums[lane] : 0;
+    const int own = s;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, s, o);
+      if (lane >= o) s += t;
+    }
+    warp_sums[lane] = s - own;
+    if (lane == 31) warp_sums[32] = s;
+  }
+  __syncthreads();
+  *total = warp_sums[32];
+  return warp_sums[wp] + x - v;
+}
+
+__global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectArgs a) {
+  __shared__ int warp_sums[33];
+  const int b = blockIdx.x, tid = threadIdx.x, nthr = blockDim.x;
+  const int nW = ws.n_windows;
+  int n = a.n_vis ? min(a.n_vis[b], ws.cap_in) : ws.cap_in;
+  if (n < 0) n = 0;
+  const int* win_off = ws.win_off + size_t(b) * (nW + 1);
+  const int* a_off = ws.a_off + size_t(b) * (nW + 1);
+  const int* tok_win = ws.tok_win + size_t(b) * ws.cap_in;
+  const int* tok_l = ws.tok_l + size_t(b) * ws.cap_in;
+  const int* a_tok = ws.a_tok + size_t(b) * ws.cap_a;
+  const int* a_win = ws.a_win + size_t(b) * ws.cap_a;
+  const float* a_f = ws.a_f + size_t(b) * ws.cap_a;
+  const int* a_best = ws.a_best + size_t(b) * ws.cap_a;
+  float* xi = ws.xi + size_t(b) * ws.cap_in;
+  int* partner = ws.partner + size_t(b) * ws.cap_in;
+  int* slot = ws.slot + size_t(b) * ws.cap_in;
+  const int* pos = a.pos ? a.pos + size_t(b) * ws.cap_in : nullptr;
+  int* dst = a.dst + size_t(b) * ws.cap_in;
+  float* weight = a.weight + size_t(b) * ws.cap_in;
+  int* grp_off = a.grp_off + size_t(b) * (a.cap_out + 1);
+  int* grp_src = a.grp_src + size_t(b) * ws.cap_in;
+  int* pos_out = a.pos_out + size_t(b) * a.cap_out;
+
+  // phase 0
+  for (int i = tid; i < n; i += nthr) {
+    float v;
+    if (a.xi_mode == LIGHTKV_XI_GIVEN) v = a.xi_in[size_t(b) * ws.cap_in + i];
+    else if (a.xi_mode == LIGHTKV_XI_UNIFORM) v = 1.0f;
+    else {
+      v = 0.f;
+      for (int h = 0; h < a.n_q_heads; ++h) v += ws.xi_h[(size_t(b) * a.n_q_heads + h) * ws.cap_in + i];
+    }
+    xi[i] = v;
+    if (a.xi_out) a.xi_out[size_t(b) * ws.cap_in + i] = v;
+    partner[i] = -1;
+  }
+  __syncthreads();
+
+  // phase 1
+  const int n_a = a_off[nW];
+  for (int e = tid; e < n_a; e += nthr) {
+    const int w = a_win[e];
+    const int e_lo = a_off[w], e_hi = a_off[w + 1];
+    const int r = removal_count(win_off[w + 1] - win_off[w], a.keep);
+    bool sel;
+    if (r <= 0) sel = false;
+    else if (r >= e_hi - e_lo) sel = true;
+    else {
+      const unsigned long long key = ((unsigned long long)orderable(a_f[e]) << 32) | (unsigned)e;
+      int rank = 0;
+      for (int e2 = e_lo; e2 < e_hi; ++e2) {
+        const unsigned long long k2 = ((unsigned long long)orderable(a_f[e2]) << 32) | (unsigned)e2;
+        rank += (k2 < key);
+      }
+      sel = rank < r;
+    }
+    if (sel && a_best[e] >= 0) partner[a_tok[e]] = a_best[e];
+  }
+  __syncthreads();
+
+  // phase 2
+  int carry = 0;
+  for (int base = 0; base < n; base += nthr) {
+    const int i = base + tid;
+    const int flag = (i < n && partner[i] < 0) ? 1 : 0;
+    int total;
+    const int ex = block_exclusive_scan(flag, warp_sums, &total);
+    if (flag) slot[i] = carry + ex;
+    carry += total;
+  }
+  const int n_out = min(carry, a.cap_out);
+  if (tid == 0) {
+    a.n_vis_out[b] = n_out;
+    if (carry > a.cap_out) set_status(a.status, LIGHTKV_STATUS_COUNT);
+  }
+  __syncthreads();
+
+  // phase 3 + 4 (sizes written where the offsets will be)
+  for (int i = tid; i < n; i += nthr) {
+    const int p = partner[i];
+    if (p >= 0) { dst[i] = slot[p]; continue; }
+    const int o = slot[i];
+    dst[i] = o;
+    if (o >= a.cap_out) continue;
+    pos_out[o] = pos ? pos[i] : i;
+    int sz = 1;
+    if (tok_l[i] & 1) {
+      const int w = tok_win[i];
+      for (int e = a_off[w]; e < a_off[w + 1]; ++e) sz += (partner[a_tok[e]] == i);
+    }
+    grp_off[o] = sz;
+  }
+  __syncthreads();
+  carry = 0;
+  for (int base = 0; base < n_out; base += nthr) {
+    const int o = base + tid;
+    const int sz = o < n_out ? grp_off[o] : 0;
+    int total;
+    const int ex = block_exclusive_scan(sz, warp_sums, &total);
+    if (o < n_out) grp_off[o] = carry + ex;
+    carry += total;
+  }
+  if (tid == 0) grp_off[n_out] = carry;
+  __syncthreads();
+
+  // phase 5
+  for (int i = tid; i < n; i += nthr) {
+    if (partner[i] >= 0) continue;
+    const int o = slot[i];
+    if (o >= a.cap_out) continue;
+    const int off = grp_off[o];
+    grp_src[off] = i;
+    int cnt = 1;
+    float den = xi[i];
+    if (tok_l[i] & 1) {
+      const int w = tok_win[i];
+      for (int e = a_off[w]; e < a_off[w + 1]; ++e) {
+        const int t = a_tok[e];
+        if (partner[t] == i) { grp_src[off + cnt++] = t; den += xi[t]; }
+      }
+    }
+    if (den >= 1e-30f) {
+      for (int c = 0; c < cnt; ++c) { const int t = grp_src[off + c]; weight[t] = xi[t] / den; }
+    } else {
+      set_status(a.status, LIGHTKV_STATUS_ZERO_WEIGHT);
+      for (int c = 0; c < cnt; ++c) weight[grp_src[off + c]] = 1.0f / (float)cnt;
+    }
+  }
+}
+
+cudaError_t launch_select_map(const LayerLaunch& L) {
+  const lightkv_layer_args_t* a = L.a;
+  SelectArgs s;
+  s.n_q_heads = L.n_q_heads; s.xi_mode = L.xi_mode; s.cap_out = L.ws.cap_out; s.keep = L.keep;
+  s.n_vis = a->n_vis; s.pos = a->pos; s.xi_in = a->xi; s.n_vis_out = a->n_vis_out; s.pos_out = a->pos_out;
+  s.dst = a->dst; s.weight = a->weight; s.grp_off = a->grp_off; s.grp_src = a->grp_src;
+  s.xi_out = a->xi_out; s.status = a->status;
+  select_map_kernel<<<L.batch, 1024, 0, L.stream>>>(L.ws, s);
+  return cudaGetLastError();
+}
+
+// =====================================================================================================
+// Weighted merge of the hidden states (Eq. "message-passing", Steps 3-5): one CTA per output row.
+// Row o of the vision block is sum over its group of weight_i * x_i in fp32, rounded once to the
+// storage type; a group of one has weight exactly 1 and is therefore copied bit-exactly.  Text rows
+// before / after the vision block are copied.  Pure 16-byte streaming loads and stores.
+// =====================================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256)
+merge_rows_kernel(const T* __restrict__ src, int64_t src_bs, int64_t src_rs,
+                  T* __restrict__ out, int64_t out_bs, int64_t out_rs,
+                  int d, int vis_begin, int n_text_after, int cap_in, int cap_out,
+                  const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
+                  const int* __restrict__ grp_off, const int* __restrict__ grp_src,
+                  const float* __restrict__ weight) {
+  constexpr int V = Vec<T>::n;
+  const int b = blockIdx.y, row = blockIdx.x;
+  const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
+  const int n_out = n_vis_out[b];
+  if (row >= vis_begin + n_out + n_text_after) return;
+  const T* sb = src + size_t(b) * src_bs;
+  T* orow = out + size_t(b) * out_bs + size_t(row) * out_rs;
+  const int chunks = d / V;
+  if (row < vis_begin || row >= vis_begin + n_out) {
+    const T* srow = sb + size_t(row < vis_begin ? row : row - n_out + n_in) * src_rs;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) st_stream16(orow + c * V, ld_stream16(srow + c * V));
+    return;
+  }
+  const int o = row - vis_begin;
+  const int* go = grp_off + size_t(b) * (cap_out + 1);
+  const int g0 = go[o], g1 = go[o + 1];
+  const int* gs = grp_src + size_t(b) * cap_in;
+  const float* wt = weight + size_t(b) * cap_in;
+  const T* vis = sb + size_t(vis_begin) * src_rs;
+  for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+    float acc[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[j] = 0.f;
+    for (int g = g0; g < g1; g += 4) {
+      uint4 v[4];
+      float wv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (g + u < g1) {
+          const int i = gs[g + u];
+          wv[u] = wt[i];
+          v[u] = ld_stream16(vis + size_t(i) * src_rs + c * V);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (g + u < g1) {
+          float f[V];
+          unpack16(v[u], f, T());
+#pragma unroll
+          for (int j = 0; j < V; ++j) acc[j] = fmaf(wv[u], f[j], acc[j]);
+        }
+      }
+    }
+    st_stream16(orow + c * V, pack16(acc, T()));
+  }
+}
+
+cudaError_t launch_merge_rows(const LayerLaunch& L) {
+  const lightkv_layer_args_t* a = L.a;
+  const int rows = a->vis_begin + L.ws.cap_out + a->n_text_after;
+  const dim3 grid(rows, L.batch);
+  if (L.dtype == LIGHTKV_BF16)
+    merge_rows_kernel<__nv_bfloat16><<<grid, 256, 0, L.stream>>>(
+        static_cast<const __nv_bfloat16*>(a->hidden), a->hidden_batch_stride, a->hidden_row_stride,
+        static_cast<__nv_bfloat16*>(a->hidden_out), a->hidden_out_batch_stride, a->hidden_out_row_stride,
+        L.hidden, a->vis_begin, a->n_text_after, L.ws.cap_in, L.ws.cap_out, a->n_vis, a->n_vis_out,
+        a->grp_off, a->grp_src, a->weight);
+  else
+    merge_rows_kernel<float><<<grid, 256, 0, L.stream>>>(
+        static_cast<const float*>(a->hidden), a->hidden_batch_stride, a->hidden_row_stride,
+        static_cast<float*>(a->hidden_out), a->hidden_out_batch_stride, a->hidden_out_row_stride,
+        L.hidden, a->vis_begin, a->n_text_after, L.ws.cap_in, L.ws.cap_out, a->n_vis, a->n_vis_out,
+        a->grp_off, a->grp_src, a->weight);
+  return cudaGetLastError();
+}
+
+// =====================================================================================================
+// K/V merge-compaction ("key and value tokens are compressed simultaneously for later layers").
+// One CTA per output token; its threads cover (K|V, head, 16-byte chunk).  The stage's merge map is
+// applied per KV head; contiguous (strided) or paged (block-table) addressing on either side.
+// =====================================================================================================
+struct KvAddr {
+  int64_t batch_stride, head_stride, row_stride, page_stride;
+  const int* table;       // nullptr = contiguous
+  int page_size, max_blocks;
+  __device__ inline int64_t token(int b, int n) const {
+    if (!table) return int64_t(b) * batch_stride + int64_t(n) * row_stride;
+    const int page = table[size_t(b) * max_blocks + n / page_size];
+    return int64_t(page) * page_stride + int64_t(n % page_size) * row_stride;
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* __restrict__ k_dst,
+                  T* __restrict__ v_dst, KvAddr sa, KvAddr da, int n_kv_heads, int dh, int vis_begin,
+                  int n_text_after, int cap_in, int cap_out, int gather,
+                  const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
+                  const int* __restrict__ grp_off, const int* __restrict__ grp_src,
+                  const float* __restrict__ weight) {
+  constexpr int V = Vec<T>::n;
+  const int b = blockIdx.y, row = blockIdx.x;
+  const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
+  const int n_out = n_vis_out[b];
+  if (row >= vis_begin + n_out + n_text_after) return;
+  const int ch = dh / V, per_kv = n_kv_heads * ch, units = 2 * per_kv;
+  const int64_t d_tok = da.token(b, row);
+  const bool text = row < vis_begin || row >= vis_begin + n_out;
+  int g0 = 0, g1 = 1;
+  int64_t s_tok = 0;
+  const int* gs = grp_src + size_t(b) * cap_in;
+  const float* wt = weight + size_t(b) * cap_in;
+  if (text) {
+    s_tok = sa.token(b, row < vis_begin ? row : row - n_out + n_in);
+  } else {
+    const int* go = grp_off + size_t(b) * (cap_out + 1);
+    g0 = go[row - vis_begin];
+    g1 = gather ? g0 + 1 : go[row - vis_begin + 1];
+    if (g1 - g0 == 1) s_tok = sa.token(b, vis_begin + gs[g0]);
+  }
+  for (int u = threadIdx.x; u < units; u += blockDim.x) {
+    const int kv = u / per_kv, rem = u - kv * per_kv, h = rem / ch, c = rem - h * ch;
+    const T* s = kv ? v_src : k_src;
+    T* dp = (kv ? v_dst : k_dst) + d_tok + int64_t(h) * da.head_stride + c * V;
+    const int64_t inner = int64_t(h) * sa.head_stride + c * V;
+    if (text || g1 - g0 == 1) {                        // copy (weight of a lone survivor is exactly 1)
+      st_stream16(dp, ld_stream16(s + s_tok + inner));
+      continue;
+    }
+    float acc[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[j] = 0.f;
+    for (int g = g0; g < g1; ++g) {
+      const int i = gs[g];
+      const float wv = wt[i];
+      float f[V];
+      unpack16(ld_stream16(s + sa.token(b, vis_begin + i) + inner), f, T());
+#pragma unroll
+      for (int j = 0; j < V; ++j) acc[j] = fmaf(wv, f[j], acc[j]);
+    }
+    st_stream16(dp, pack16(acc, T()));
+  }
+}
+
+cudaError_t launch_kv_compact(const KvLaunch& K) {
+  const lightkv_kv_args_t* a = K.a;
+  KvAddr sa{a->src_batch_stride, a->src_head_stride, a->src_row_stride, a->src_page_stride,
+            a->page_size > 0 ? a->src_block_table : nullptr, a->page_size, a->max_blocks};
+  KvAddr da{a->dst_batch_stride, a->dst_head_stride, a->dst_row_stride, a->dst_page_stride,
+            a->page_size > 0 ? a->dst_block_table : nullptr, a->page_size, a->max_blocks};
+  const dim3 grid(a->vis_begin + K.cap_out + a->n_text_after, K.batch);
+  const int gather = a->mode == LIGHTKV_KV_GATHER;
+  if (K.dtype == LIGHTKV_BF16)
+    kv_compact_kernel<__nv_bfloat16><<<grid, 256, 0, K.stream>>>(
+        static_cast<const __nv_bfloat16*>(a->k_src), static_cast<const __nv_bfloat16*>(a->v_src),
+        static_cast<__nv_bfloat16*>(a->k_dst), static_cast<__nv_bfloat16*>(a->v_dst), sa, da, K.n_kv_heads,
+        K.head_dim, a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, a->n_vis, a->n_vis_out,
+        a->grp_off, a->grp_src, a->weight);
+  else
+    kv_compact_kernel<float><<<grid, 256, 0, K.stream>>>(
+        static_cast<const float*>(a->k_src), static_cast<const float*>(a->v_src),
+        static_cast<float*>(a->k_dst), static_cast<float*>(a->v_dst), sa, da, K.n_kv_heads, K.head_dim,
+        a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, a->n_vis, a->n_vis_out, a->grp_off,
+        a->grp_src, a->weight);
+  return cudaGetLastError();
+}
+
+}  // namespace lkv

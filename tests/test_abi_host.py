@@ -1,0 +1,155 @@
+"""CPU-only checks of the C ABI: the library loads, exports every declared symbol, and rejects bad
+arguments on the host before anything is launched (no GPU needed)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    entry.build()
+    import paper_2605_00789_b200 as pkg
+    return pkg
+
+
+def test_every_declared_symbol_is_exported(L):
+    header = open(os.path.join(ROOT, "include", "lightkv.h")).read()
+    declared = set(re.findall(r"\b(lightkv_[a-z_]+)\s*\(", header))
+    assert declared == set(L.lightkv.EXPORTS)
+    lib = L.library()
+    for name in declared:
+        assert getattr(lib, name) is not None
+    assert L.version() == 100
+    assert L.status_string(0) == "ok" and "workspace" in L.status_string(-3)
+
+
+def test_struct_layouts_match_the_header(L, tmp_path):
+    """Ask the C compiler for the size of every struct and the offset of its last field."""
+    import subprocess
+    src = tmp_path / "layout.c"
+    src.write_text('''#include <stdio.h>
+#include <stddef.h>
+#include "lightkv.h"
+int main(void) {
+  printf("%zu %zu\\n", sizeof(lightkv_config_t), offsetof(lightkv_config_t, engine));
+  printf("%zu %zu\\n", sizeof(lightkv_stage_info_t), offsetof(lightkv_stage_info_t, workspace_bytes));
+  printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, stream));
+  printf("%zu %zu\\n", sizeof(lightkv_kv_args_t), offsetof(lightkv_kv_args_t, stream));
+  return 0;
+}
+''')
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    rows = [tuple(int(v) for v in line.split()) for line in subprocess.check_output([str(exe)]).decode().splitlines()]
+    k = L.lightkv
+    got = [(C.sizeof(k._Config), k._Config.engine.offset),
+           (C.sizeof(k._StageInfo), k._StageInfo.workspace_bytes.offset),
+           (C.sizeof(k._LayerArgs), k._LayerArgs.stream.offset),
+           (C.sizeof(k._KvArgs), k._KvArgs.stream.offset)]
+    assert got == rows
+
+
+def _plan(L, **kw):
+    args = dict(batch=2, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=16, n_layers=8, tiles=[(6, 6)],
+                layers=[2, 4], windows=[2, 1], keep=[0.5, 0.5], max_text=16)
+    args.update(kw)
+    return L.Plan(**args)
+
+
+def test_plan_counts_and_retention(L):
+    p = _plan(L, tiles=[(24, 24)], layers=[12, 18, 24], windows=[4, 2, 1], keep=[0.5] * 3, n_layers=32,
+              hidden=4096, n_q_heads=32, n_kv_heads=32, head_dim=128, batch=1, max_text=64)
+    caps = [(p.stage_info(s).cap_in, p.stage_info(s).cap_out, p.stage_info(s).n_windows,
+             p.stage_info(s).counts_exact) for s in range(3)]
+    assert caps == [(576, 288, 16, 1), (288, 144, 4, 1), (144, 72, 1, 1)]
+    assert p.retention() == pytest.approx(0.546875)
+    p = _plan(L, tiles=[(24, 24)], layers=[15, 23, 31], windows=[4, 2, 1], keep=[0.5] * 3, n_layers=40)
+    assert p.retention() == pytest.approx(0.553125)
+    p = _plan(L, tiles=[(24, 24)], layers=[10, 20, 30], windows=[4, 2, 1], keep=[0.5] * 3, n_layers=40)
+    assert p.retention() == pytest.approx(0.46875)
+    # data-dependent counts: capacities are upper bounds
+    p = _plan(L, tiles=[(24, 24)], layers=[12], windows=[4], keep=[0.55], n_layers=32)
+    info = p.stage_info(0)
+    assert info.counts_exact == 0 and 320 <= info.cap_out <= 576 and info.workspace_bytes > 0
+    # odd windows (9 tokens) under keep 0.5 leave one data-dependent A node per window
+    p = _plan(L)
+    assert p.stage_info(0).counts_exact == 0 and p.stage_info(0).cap_out >= 20
+
+
+@pytest.mark.parametrize("kw", [
+    dict(batch=0), dict(hidden=65), dict(head_dim=12), dict(n_q_heads=3), dict(keep=[0.4, 0.5]),
+    dict(keep=[0.5, 1.5]), dict(windows=[7, 1]), dict(windows=[0, 1]), dict(layers=[4, 2]),
+    dict(layers=[2, 9]), dict(tiles=[(0, 6)]), dict(dtype=7), dict(xi_mode=9), dict(engine=5),
+])
+def test_plan_rejects_bad_configs(L, kw):
+    with pytest.raises(L.LightKVError, match="invalid argument"):
+        _plan(L, **kw)
+
+
+def test_plan_unsupported(L):
+    with pytest.raises(L.LightKVError, match="unsupported"):
+        _plan(L, tiles=[(6, 6)] * 33)
+    with pytest.raises(L.LightKVError, match="unsupported"):
+        _plan(L, tiles=[(64, 64)], windows=[64, 1])
+
+
+def test_calls_reject_bad_arguments_before_any_launch(L):
+    p = _plan(L)
+    lib = L.library()
+    a = L.lightkv._LayerArgs()
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # struct_size
+    a.struct_size = C.sizeof(a)
+    a.stage = 5
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # stage
+    a.stage = 0
+    a.vis_begin, a.text_end = 4, 9
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # J outside the text rows
+    a.text_end = 4
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # NULL buffers
+    for f in ("hidden", "n_vis_out", "pos_out", "dst", "weight", "grp_off", "grp_src", "workspace"):
+        setattr(a, f, 0x1000)
+    a.hidden_out = 0x2000
+    a.hidden_row_stride = a.hidden_out_row_stride = 64
+    a.hidden_batch_stride = a.hidden_out_batch_stride = 64 * 64
+    a.workspace_bytes = 16
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -3            # workspace too small
+    a.workspace_bytes = 1 << 30
+    a.hidden = 0x1008
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # misaligned rows
+    a.hidden = 0x1000
+    a.hidden_row_stride = 60
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # row stride below hidden
+    a.hidden_row_stride = 64
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # ATTN_FULL without q / k
+    assert lib.lightkv_compress_layer(None, C.byref(a)) == -1
+
+    kv = L.lightkv._KvArgs()
+    assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1
+    kv.struct_size = C.sizeof(kv)
+    kv.mode = 3
+    assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1
+    kv.mode = 0
+    for f in ("n_vis_out", "grp_off", "grp_src", "weight", "k_src", "v_src"):
+        setattr(kv, f, 0x1000)
+    kv.k_dst = kv.v_dst = 0x1000
+    kv.src_row_stride = kv.dst_row_stride = 16
+    assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1               # in place is not supported
+    kv.k_dst = kv.v_dst = 0x3000
+    kv.page_size = 16
+    assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1               # paged without block tables
+    assert lib.lightkv_plan_stage_info(p.handle, 9, C.byref(L.lightkv._StageInfo())) == -1
+    assert lib.lightkv_plan_retention(None) < 0
+
+
+def test_missing_library_fails_loudly(L, monkeypatch):
+    from paper_2605_00789_b200 import lightkv
+    monkeypatch.setattr(lightkv, "_LIB", None)
+    monkeypatch.setattr(lightkv, "_HERE", "/nonexistent")
+    with pytest.raises(L.LightKVError, match="missing"):
+        lightkv.library()

@@ -1,0 +1,148 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on seeded synthetic inputs.
+
+Index sets (survivors, dst, positions, counts, group lists) must be bit-exact on inputs whose
+selection margins are >= 1e-3; merged hidden states and K/V within max-abs 2e-2 and relative 1e-2
+(bf16 storage, fp32 accumulation) or 1e-5 relative (fp32 mode)."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import lightkv_synth as S
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    import torch
+    import __graft_entry__ as entry
+    assert torch.cuda.is_available()
+    entry.build()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("engine", ["simt", "auto"])
+@pytest.mark.parametrize("xi_mode", ["attn", "lse", "given", "uniform"])
+def test_tiny_schedule(dtype, engine, xi_mode):
+    stats = H.run_schedule(S.workload("tiny"), dtype=dtype, xi_mode=xi_mode, engine=engine)
+    assert [s["n_out"] for s in stats] == [[20, 20], [15, 15], [8, 8]]
+
+
+@pytest.mark.parametrize("dtype,engine", [("bf16", "simt"), ("bf16", "auto"), ("fp32", "simt")])
+def test_small_ragged_multitile_gqa(dtype, engine):
+    # two tiles of different shape, windows that do not divide the grid, GQA, keep 0.55 / 0.6 / 0.5
+    H.run_schedule(S.workload("small"), dtype=dtype, engine=engine)
+
+
+@pytest.mark.parametrize("kv_mode,paged", [("gather", 0), ("merge", 16), ("gather", 16), ("merge", 5)])
+def test_small_kv_modes_and_paged_cache(kv_mode, paged):
+    H.run_schedule(S.workload("small"), kv_mode=kv_mode, paged=paged, stages=[0])
+
+
+@pytest.mark.parametrize("w", [4, 6, 1])
+@pytest.mark.parametrize("engine", ["simt", "auto"])
+def test_cfg0_single_step(w, engine):
+    wl = dataclasses.replace(S.workload("cfg0"), windows=(w,))
+    stats = H.run_schedule(wl, engine=engine)
+    assert stats[0]["n_out"] == [{4: 320, 6: 324, 1: 317}[w]]
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg1r"])
+def test_cfg1_full_schedule(name):
+    stats = H.run_schedule(S.workload(name))
+    if name == "cfg1":
+        assert [s["n_out"] for s in stats] == [[288], [144], [72]]
+
+
+def test_cfg0_fp32_mode():
+    H.run_schedule(dataclasses.replace(S.workload("cfg0"), hidden=1024, n_q_heads=8, n_kv_heads=8), dtype="fp32")
+
+
+def test_text_after_and_prompt_subrange():
+    wl = S.workload("small")
+    plan = H.make_plan(wl)
+    inp = H.prepare_stage(wl, 0)
+    # move the last 4 text rows behind the vision block: [15 text | vision | 4 text], J = [2, 12)
+    vb, after = wl.n_text - 4, 4
+    for key in ("hidden", "q", "k", "v"):
+        a = inp[key]
+        axis = 1 if key == "hidden" else 2
+        a = np.concatenate([np.take(a, range(0, vb), axis), np.take(a, range(wl.n_text, a.shape[axis]), axis),
+                            np.take(a, range(vb, wl.n_text), axis)], axis)
+        inp[key] = np.ascontiguousarray(a)
+    inp["vis_begin"] = vb
+    assert len(set(inp["n_vis"])) == 1        # full grids: every sample has the same length here
+    gpu = H.gpu_stage(plan, wl, 0, inp, n_text_after=after, text_range=(2, 12))
+    ref = H.oracle_stage(wl, 0, inp, n_text_after=after, text_range=(2, 12))
+    H.compare_stage(wl, 0, inp, ref, gpu, n_text_after=after)
+    for b, r in enumerate(ref):
+        n_out = int(r["n_out"])
+        np.testing.assert_array_equal(gpu["hidden_out"][b, vb + n_out:vb + n_out + after],
+                                      inp["hidden"][b, vb + int(inp["n_vis"][b]):][:after])
+
+
+def test_ragged_batch_and_empty_sample():
+    wl = S.workload("small")
+    plan = H.make_plan(wl)
+    full = np.arange(wl.n_vis, dtype=np.int32)
+    rng = np.random.default_rng(5)
+    pos = [full, np.sort(rng.choice(full, 97, replace=False)).astype(np.int32), full[:0]]
+    inp = H.prepare_stage(wl, 0, pos)
+    gpu = H.gpu_stage(plan, wl, 0, inp)
+    ref = H.oracle_stage(wl, 0, inp)
+    H.compare_stage(wl, 0, inp, ref, gpu)
+    assert int(gpu["n_vis_out"][2]) == 0
+
+
+def test_keep_one_is_identity_on_device():
+    wl = dataclasses.replace(S.workload("small"), keep=(1.0, 1.0, 1.0))
+    plan = H.make_plan(wl)
+    inp = H.prepare_stage(wl, 0, repair=False)
+    gpu = H.gpu_stage(plan, wl, 0, inp)
+    n = wl.n_vis
+    assert (gpu["n_vis_out"] == n).all()
+    np.testing.assert_array_equal(gpu["hidden_out"][:, :wl.n_text + n], inp["hidden"])
+    np.testing.assert_array_equal(gpu["k_out"][:, :, :wl.n_text + n], inp["k"])
+    np.testing.assert_array_equal(gpu["dst"][:, :n], np.tile(np.arange(n), (wl.batch, 1)))
+    assert (gpu["weight"][:, :n] == 1.0).all()
+
+
+def test_device_status_word_flags_unsorted_positions():
+    wl = S.workload("tiny")
+    plan = H.make_plan(wl, xi_mode="uniform")
+    inp = H.prepare_stage(wl, 0, repair=False)
+    inp["pos"][1, [3, 4]] = inp["pos"][1, [4, 3]]
+    gpu = H.gpu_stage(plan, wl, 0, inp, xi_mode="uniform")
+    assert int(gpu["status"][0]) & 1
+
+
+def test_run_to_run_bit_repeatability():
+    wl = S.workload("small")
+    plan = H.make_plan(wl)
+    inp = H.prepare_stage(wl, 0, repair=False)
+    a = H.gpu_stage(plan, wl, 0, inp)
+    b = H.gpu_stage(plan, wl, 0, inp)
+    for key in ("hidden_out", "k_out", "v_out", "weight", "xi_out", "dst", "grp_src", "grp_off", "pos_out"):
+        np.testing.assert_array_equal(a[key], b[key])
+
+
+# ---- full benchmark shapes, compared on the samples the oracle can finish in seconds -----------------
+
+def test_cfg2_full_size_sampled():
+    stats = H.run_schedule(S.workload("cfg2"), oracle_samples=[0, 5])
+    assert [s["n_out"] for s in stats] == [[1440] * 8, [720] * 8, [360] * 8]
+
+
+def test_cfg3_first_stage_sampled():
+    H.run_schedule(S.workload("cfg3"), stages=[0], oracle_samples=[0, 31])
+
+
+def test_cfg4_gqa_video_first_stage_sampled():
+    H.run_schedule(S.workload("cfg4"), stages=[0], oracle_samples=[1])
+
+
+def test_cfg4g_large_windows_uniform_xi():
+    # windows of 512 tokens: exercises the multi-chunk B loop of the FD kernels
+    H.run_schedule(S.workload("cfg4g"), xi_mode="uniform", stages=[0], oracle_samples=[0])
