@@ -196,7 +196,7 @@ def compare_stage(wl, stage, inp, ref, gpu, dtype="bf16", kv_mode="merge", n_tex
         stats["hidden_max_abs"] = max(stats["hidden_max_abs"], ma)
         stats["hidden_rel"] = max(stats["hidden_rel"], rel)
         # tokens that were not merged are copied bit-exactly
-        single = np.array([off[o + 1] - off[o] == 1 for o in range(n_out)])
+        single = np.array([off[o + 1] - off[o] == 1 for o in range(n_out)], dtype=bool)
         np.testing.assert_array_equal(gpu["hidden_out"][b, vb:vb + n_out][single],
                                       inp["hidden"][b, vb + r["survivor"]][single])
         np.testing.assert_array_equal(gpu["hidden_out"][b, :vb], inp["hidden"][b, :vb])
