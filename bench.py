@@ -1,0 +1,404 @@
+#!/usr/bin/env python
+"""Benchmark of the LightKV compression hot path on B200 (one JSON line on stdout).
+
+A step = one pass of the whole hot path over one batch: for every stage of the workload's schedule,
+lightkv_compress_layer (window build, xi, FD + best partner, selection + merge map, hidden merge) and
+lightkv_compact_kv on that layer's K/V, chained through the surviving positions on the device.
+Inputs are seeded synthetic tensors (lightkv_synth), regenerated per compression layer and resident
+in HBM before the timed region.  `value` is vision tokens entering compression stages per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+
+N > 1 (under torchrun): every rank compresses its own batch (no data-path collective, weak scaling);
+the time is the max over ranks.  --impl reference times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import lightkv_synth as S  # noqa: E402
+
+KERNELS = ("window_build", "xi", "fd_best_partner", "select_map", "merge_hidden", "kv_compact")
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
+# keyed by (workload, kernel); null until a capture exists for that pair.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.file = index, None, None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------ workload
+
+def build_inputs(wl, plan, L, torch, device, sample_offset):
+    """Generate every stage's inputs on the host (pinned) and upload them.  Stage i+1 is sampled at the
+    positions that survive stage i (taken from one untimed run of the library itself)."""
+    samples = [sample_offset + b for b in range(wl.batch)]
+    stages, pos = [], None
+    for st in range(wl.n_stages):
+        info = plan.stage_info(st)
+        inp = S.make_layer_inputs(wl, st, pos, samples=samples)
+        host, dev = {}, {}
+        for name in ("hidden", "q", "k", "v"):
+            t = torch.from_numpy(S.bf16_bits(inp[name]).view(np.int16)).view(torch.bfloat16).pin_memory()
+            host[name] = t
+            dev[name] = t.to(device, non_blocking=True)
+        n_seq = host["hidden"].shape[1]
+        pos_pad = np.full((wl.batch, info.cap_in), -1, dtype=np.int32)
+        pos_pad[:, :inp["pos"].shape[1]] = inp["pos"]
+        dev["pos"] = torch.from_numpy(pos_pad).to(device)
+        dev["n_vis"] = torch.from_numpy(inp["n_vis"]).to(device)
+        n_seq_out = wl.n_text + info.cap_out
+        out = L.StageBuffers(plan, st, n_seq_out, device)
+        k_dst = torch.empty((wl.batch, wl.n_kv_heads, n_seq_out, wl.head_dim), dtype=torch.bfloat16, device=device)
+        v_dst = torch.empty_like(k_dst)
+        host_out = {"hidden": torch.empty(out.hidden_out.shape, dtype=torch.bfloat16).pin_memory(),
+                    "k": torch.empty(k_dst.shape, dtype=torch.bfloat16).pin_memory(),
+                    "v": torch.empty(k_dst.shape, dtype=torch.bfloat16).pin_memory(),
+                    "n_vis_out": torch.empty((wl.batch,), dtype=torch.int32).pin_memory(),
+                    "pos_out": torch.empty(out.pos_out.shape, dtype=torch.int32).pin_memory()}
+        stg = dict(info=info, host=host, dev=dev, out=out, k_dst=k_dst, v_dst=v_dst, host_out=host_out,
+                   n_vis=inp["n_vis"].copy(), n_seq=n_seq, n_seq_out=n_seq_out)
+        stages.append(stg)
+        run_stage(L, plan, wl, st, stg, stg["dev"]["pos"], stg["dev"]["n_vis"])
+        torch.cuda.synchronize()
+        n_out = out.n_vis_out.cpu().numpy()
+        pos_out = out.pos_out.cpu().numpy()
+        stg["n_out"] = n_out.copy()
+        pos = [pos_out[b, :n_out[b]] for b in range(wl.batch)]
+        if int(out.status.item()) != 0:
+            raise RuntimeError(f"device status word {int(out.status.item())} at stage {st}")
+    return stages
+
+
+def run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None):
+    d = stg["dev"]
+    L.compress_layer(plan, st, d["hidden"], stg["out"], vis_begin=wl.n_text, q=d["q"], k=d["k"], n_vis=n_vis,
+                     pos=pos, trace_events=trace)
+    L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
+                 n_vis=n_vis)
+
+
+def run_step(L, plan, wl, stages, traces=None, kv_events=None):
+    """The whole hot path once; stage i+1 reads positions and counts stage i left on the device."""
+    pos, n_vis = stages[0]["dev"]["pos"], stages[0]["dev"]["n_vis"]
+    for st, stg in enumerate(stages):
+        run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None if traces is None else traces[st])
+        if kv_events is not None:
+            kv_events[st].record()
+        pos, n_vis = stg["out"].pos_out, stg["out"].n_vis_out
+
+
+def algorithmic_work(wl, stages):
+    """Per kernel, summed over the stages of one step: algorithmic bytes (HBM streams) or flops (xi)."""
+    e = 2  # bf16
+    work = {k: 0.0 for k in KERNELS}
+    nt = wl.n_text
+    for stg in stages:
+        n_in = stg["n_vis"].astype(np.float64)
+        n_out = stg["n_out"].astype(np.float64)
+        # xi, ATTN_FULL: 2*dh flops per (head, query, visible key); query t sees n_text + t + 1 keys
+        work["xi"] += float((2.0 * wl.n_q_heads * wl.head_dim * (n_in * (nt + 1) + n_in * (n_in - 1) / 2)).sum())
+        # FD: one read of the vision rows (+ 8 bytes of keys per A node)
+        work["fd_best_partner"] += float((n_in * wl.hidden * e + 4 * n_in).sum())
+        # hidden merge: every input row read once, every output row written once
+        work["merge_hidden"] += float(((nt + n_in) * wl.hidden * e + (nt + n_out) * wl.hidden * e).sum())
+        # K/V: same for K and V, all KV heads
+        work["kv_compact"] += float((2 * wl.n_kv_heads * wl.head_dim * e * ((nt + n_in) + (nt + n_out))).sum())
+        work["window_build"] += float((n_in * 4 * 5).sum())
+        work["select_map"] += float((n_in * 4 * 10).sum())
+    return work
+
+
+def oracle_sample_step(wl, full_schedule=True):
+    """The CPU oracle on a bounded sample of the workload: sample 0 through the schedule (or its last
+    stage only).  Returns (seconds, vision tokens entering the stages it ran)."""
+    from oracle import lightkv_oracle as O
+    t_total, tokens = 0.0, 0
+    pos = None
+    stage_list = range(wl.n_stages)
+    for st in stage_list:
+        inp = S.make_layer_inputs(wl, st, pos, samples=[0])
+        if not full_schedule and st < wl.n_stages - 1:
+            # advance the positions cheaply with uniform xi (not timed)
+            res = O.compress_layer(inp["hidden"], None, None, inp["pos"], inp["n_vis"], inp["vis_begin"], wl.tiles,
+                                   wl.windows[st], wl.keep[st])
+            pos = [res[0]["pos_out"]]
+            continue
+        t0 = time.perf_counter()
+        res = O.compress_layer(inp["hidden"], inp["q"], inp["k"], inp["pos"], inp["n_vis"], inp["vis_begin"],
+                               wl.tiles, wl.windows[st], wl.keep[st])
+        r = res[0]
+        nv = int(inp["n_vis"][0])
+        for name in ("k", "v"):
+            O.compact_kv(inp[name][0][:, :inp["vis_begin"] + nv], inp["vis_begin"], nv, r["dst"], r["weight"],
+                         r["survivor"], "merge")
+        t_total += time.perf_counter() - t0
+        tokens += nv
+        pos = [r["pos_out"]]
+    return t_total, tokens
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------------------------ main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg2", choices=sorted(S.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = S.workload(args.workload)
+    metric, unit = "vision_tokens_compressed_per_s", "tokens/s"
+    config = {"workload": f"{wl.name}: {wl.n_stages}-stage schedule layers={list(wl.layers)} windows={list(wl.windows)} "
+                          f"keep={list(wl.keep)}, batch {wl.batch}, {wl.n_vis} vision + {wl.n_text} text tokens, "
+                          f"hidden {wl.hidden}, {wl.n_q_heads}q/{wl.n_kv_heads}kv heads x {wl.head_dim}, "
+                          f"xi from full causal attention, K/V merge",
+              "l2": "inputs larger than L2 (every stage streams > 126 MB)", "batch_per_gpu": wl.batch}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        budget = 150.0
+        t_last, tok_last = oracle_sample_step(wl, full_schedule=False)
+        full = t_last * 12 * (args.steps + args.warmup) < budget     # the full schedule costs ~10x its last stage
+        times, tokens = [], 0
+        for i in range(args.warmup + args.steps):
+            t, tokens = oracle_sample_step(wl, full_schedule=full)
+            if i >= args.warmup:
+                times.append(t)
+        ms = 1e3 * sum(times) / len(times)
+        value = tokens / (ms / 1e3)
+        sample = f"sample 0 of {wl.batch}, " + ("all stages" if full else "last stage only") + f" ({tokens} vision tokens per step)"
+        line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": value, "unit": unit, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+                "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    if local_rank == 0:
+        entry.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2605_00789_b200 as L
+
+    plan = L.Plan(wl.batch, wl.hidden, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_layers, wl.tiles, wl.layers,
+                  wl.windows, wl.keep, wl.n_text, dtype=L.BF16, xi_mode=L.XI_ATTN_FULL,
+                  engine=L.ENGINE_AUTO if args.engine == "auto" else L.ENGINE_SIMT)
+    stages = build_inputs(wl, plan, L, torch, device, sample_offset=rank * wl.batch)
+    tokens_per_step = int(sum(int(s["n_vis"].sum()) for s in stages))
+    n_stages = len(stages)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        run_step(L, plan, wl, stages)
+    # per-kernel events inside the timed region: TRACE_EVENTS per (step, stage) + one after compact_kv
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()                    # torch creates the CUDA event lazily; the C ABI needs a live handle
+        return e
+    traces = [[[ev() for _ in range(L.TRACE_EVENTS)] for _ in range(n_stages)] for _ in range(args.steps)]
+    kv_ev = [[ev() for _ in range(n_stages)] for _ in range(args.steps)]
+    t_begin, t_end = ev(), ev()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t_begin.record()
+    for i in range(args.steps):
+        run_step(L, plan, wl, stages, traces[i], kv_ev[i])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = t_begin.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([ms_total], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * tokens_per_step / (ms_step / 1e3)
+
+    ktime = {k: 0.0 for k in KERNELS}       # ms per step, summed over stages
+    for i in range(args.steps):
+        for st in range(n_stages):
+            e = traces[i][st]
+            for j, name in enumerate(L.TRACE_NAMES):
+                ktime[name] += e[j].elapsed_time(e[j + 1])
+            ktime["kv_compact"] += e[-1].elapsed_time(kv_ev[i][st])
+    ktime = {k: v / args.steps for k, v in ktime.items()}
+    work = algorithmic_work(wl, stages)
+    peaks = measured_peaks()
+    kernels = {}
+    for k in KERNELS:
+        sec = ktime[k] / 1e3
+        if k == "xi":
+            ach, peak, u, bound = work[k] / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", "tensor"
+        else:
+            ach, peak, u, bound = work[k] / sec / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+        kernels[k] = {"ms_per_step": round(ktime[k], 4), "share": round(ktime[k] / sum(ktime.values()), 4),
+                      "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": u, "frac": round(ach / peak, 4)}
+    top = max(KERNELS, key=lambda k: ktime[k])
+    roofline = {"kernel": top, "bound": kernels[top]["bound"], "achieved": kernels[top]["achieved"],
+                "peak": kernels[top]["peak"], "unit": kernels[top]["unit"], "frac": kernels[top]["frac"],
+                "traffic": NCU_TRAFFIC_BYTES.get((wl.name, top)), "peak_source": f"of {peaks['source']}",
+                "launches_per_step": n_stages}
+
+    # end to end through the public API with host buffers: H2D of every stage's inputs from pinned
+    # memory, the step, D2H of every stage's results
+    e2e = None
+    if not args.no_e2e:
+        h2d = sum(t.numel() * t.element_size() for s in stages for t in s["host"].values())
+        d2h = sum(t.numel() * t.element_size() for s in stages for t in s["host_out"].values())
+
+        def e2e_step():
+            for st, s in enumerate(stages):
+                for name, t in s["host"].items():
+                    s["dev"][name].copy_(t, non_blocking=True)
+            run_step(L, plan, wl, stages)
+            for s in stages:
+                s["host_out"]["hidden"].copy_(s["out"].hidden_out, non_blocking=True)
+                s["host_out"]["k"].copy_(s["k_dst"], non_blocking=True)
+                s["host_out"]["v"].copy_(s["v_dst"], non_blocking=True)
+                s["host_out"]["n_vis_out"].copy_(s["out"].n_vis_out, non_blocking=True)
+                s["host_out"]["pos_out"].copy_(s["out"].pos_out, non_blocking=True)
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        ms_e2e = a.elapsed_time(b) / e2e_steps
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": world * tokens_per_step / (ms_e2e / 1e3), "unit": unit, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        t, tok = oracle_sample_step(wl, full_schedule=True)
+        cpu = {"value": tok / t, "unit": unit, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"sample 0 of {wl.batch}, all {n_stages} stages ({tok} vision tokens, {t:.1f} s)"}
+
+    if rank == 0:
+        launches_per_step = n_stages * 6
+        line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
+                "us_per_compression_layer": 1e3 * ms_step / n_stages,
+                "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+                "gpu_launches": launches_per_step * args.steps,
+                "engine": {st: int(plan.stage_info(st).uses_tensor_cores) for st in range(n_stages)}}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -166,7 +166,14 @@ typedef struct {
   void*   workspace;               /* DEVICE, 256-byte aligned */
   size_t  workspace_bytes;
   void*   stream;                  /* cudaStream_t */
+  void**  trace_events;            /* HOST array of LIGHTKV_TRACE_EVENTS cudaEvent_t created by the caller,
+                                      or NULL.  Event 0 is recorded on the stream before the first kernel,
+                                      event i after kernel i: 1 window build, 2 xi, 3 FD + best partner,
+                                      4 selection + merge map, 5 hidden-state merge (a kernel the mode skips
+                                      still gets its event).  For per-kernel timing. */
 } lightkv_layer_args_t;
+
+#define LIGHTKV_TRACE_EVENTS 6
 
 /* Enqueue window build, xi, FD + best partner, selection + merge map and the
  * weighted merge of the hidden states.  Errors: INVALID_ARG, WORKSPACE (too

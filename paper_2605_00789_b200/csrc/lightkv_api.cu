@@ -250,18 +250,22 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
   L.head_dim = c.head_dim; L.dtype = c.dtype; L.xi_mode = c.xi_mode; L.keep = s.keep; L.geo = s.geo;
   L.ws = bind_workspace(s, a->workspace); L.a = a; L.stream = static_cast<cudaStream_t>(a->stream);
 
-  cudaError_t e;
-  if ((e = launch_window_build(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+  cudaEvent_t* ev = reinterpret_cast<cudaEvent_t*>(a->trace_events);
+  auto mark = [&](int i) { return ev ? cudaEventRecord(ev[i], L.stream) : cudaSuccess; };
+  if (mark(0) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+  if (launch_window_build(L) != cudaSuccess || mark(1) != cudaSuccess) return LIGHTKV_ERR_CUDA;
   if (attn) {
     const bool tc = s.use_tc && c.xi_mode == LIGHTKV_XI_ATTN_FULL && tc_xi_supported(c.head_dim);
-    if ((e = tc ? launch_xi_tc(L) : launch_xi_simt(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    if ((tc ? launch_xi_tc(L) : launch_xi_simt(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
   }
+  if (mark(2) != cudaSuccess) return LIGHTKV_ERR_CUDA;
   {
     const bool tc = s.use_tc && tc_fd_supported(c.hidden);
-    if ((e = tc ? launch_fd_tc(L) : launch_fd_simt(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    if ((tc ? launch_fd_tc(L) : launch_fd_simt(L)) != cudaSuccess || mark(3) != cudaSuccess)
+      return LIGHTKV_ERR_CUDA;
   }
-  if ((e = launch_select_map(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
-  if ((e = launch_merge_rows(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+  if (launch_select_map(L) != cudaSuccess || mark(4) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+  if (launch_merge_rows(L) != cudaSuccess || mark(5) != cudaSuccess) return LIGHTKV_ERR_CUDA;
   return LIGHTKV_OK;
 }
 

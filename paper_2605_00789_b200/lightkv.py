@@ -58,7 +58,12 @@ class _LayerArgs(C.Structure):
                 ("n_vis_out", C.c_void_p), ("pos_out", C.c_void_p), ("dst", C.c_void_p),
                 ("weight", C.c_void_p), ("grp_off", C.c_void_p), ("grp_src", C.c_void_p),
                 ("xi_out", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
-                ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p)]
+                ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p),
+                ("trace_events", C.POINTER(C.c_void_p))]
+
+
+TRACE_EVENTS = 6
+TRACE_NAMES = ("window_build", "xi", "fd_best_partner", "select_map", "merge_hidden")
 
 
 class _KvArgs(C.Structure):
@@ -206,7 +211,8 @@ def _stream_handle(stream) -> int:
 
 def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin: int,
                    n_text_after: int = 0, text_begin: int = 0, text_end: Optional[int] = None,
-                   q=None, k=None, lse=None, xi=None, n_vis=None, pos=None, stream=None) -> None:
+                   q=None, k=None, lse=None, xi=None, n_vis=None, pos=None, stream=None,
+                   trace_events=None) -> None:
     """lightkv_compress_layer.  hidden [B,N,d]; q [B,H,N,dh]; k [B,H_kv,N,dh] (any strides with a
     contiguous last dimension); lse [B,H,N] fp32; xi [B,cap_in] fp32; n_vis [B] int32; pos [B,cap_in] int32."""
     a = _LayerArgs()
@@ -227,6 +233,9 @@ def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_beg
     a.grp_off, a.grp_src, a.xi_out, a.status = _ptr(out.grp_off), _ptr(out.grp_src), _ptr(out.xi_out), _ptr(out.status)
     a.workspace, a.workspace_bytes = out.workspace_ptr(), out.info.workspace_bytes
     a.stream = _stream_handle(stream)
+    if trace_events is not None:      # TRACE_EVENTS torch.cuda.Event objects (enable_timing=True), already created
+        assert len(trace_events) == TRACE_EVENTS
+        a.trace_events = (C.c_void_p * TRACE_EVENTS)(*[e.cuda_event for e in trace_events])
     _check(library().lightkv_compress_layer(plan.handle, C.byref(a)), "lightkv_compress_layer")
 
 
