@@ -171,6 +171,8 @@ typedef struct {
                                       event i after kernel i: 1 window build, 2 xi, 3 FD + best partner,
                                       4 selection + merge map, 5 hidden-state merge (a kernel the mode skips
                                       still gets its event).  For per-kernel timing. */
+  int32_t seq_rows;                /* rows every (sample, head) slice of q / k really holds (tensor-map
+                                      bound of the TMA loads); 0 = vis_begin + cap_in + n_text_after */
 } lightkv_layer_args_t;
 
 #define LIGHTKV_TRACE_EVENTS 6

@@ -1,9 +1,251 @@
-// liblightkv kernels, part 2: tcgen05 tensor-core contractions (placeholder until the kernels land).
+// liblightkv kernels, part 2: tcgen05 tensor-core contractions fed by TMA (sm_100a).
 #include "launch.h"
+#include "tc_common.cuh"
 
 namespace lkv {
+
+using namespace tc;
+
+// ------------------------------------------------------------------------------------------------------
+// Host: tensor maps.  cuTensorMapEncodeTiled is fetched through the runtime so that the library does not
+// link against libcuda.
+// ------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [batch, heads, rows, width] with element strides (width contiguous); box = 64 x box_rows
+// elements, 128-byte swizzle.
+static bool make_map_bhnd(CUtensorMap* map, const void* base, int width, int rows, int heads, int batch,
+                          int64_t row_stride, int64_t head_stride, int64_t batch_stride, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)width, (cuuint64_t)rows, (cuuint64_t)heads, (cuuint64_t)batch};
+  const cuuint64_t strides[3] = {(cuuint64_t)row_stride * 2, (cuuint64_t)head_stride * 2,
+                                 (cuuint64_t)(batch > 1 ? batch_stride : head_stride * heads) * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ======================================================================================================
+// xi per head on tensor cores (Eq. "attention-factor" over the causal softmax rows of Eq.
+// "attention-matrix").
+//
+// One CTA per (tile of 128 vision queries, head, sample); two CTAs share an SM.  Warp 0 streams the Q tile
+// once and the K tiles through a 2-stage ring with TMA; warp 1 issues S = Q K^T (128 x 128 x dh, bf16 ->
+// fp32) into one of two TMEM accumulators; warps 2-5 own one query row per thread (= TMEM lane), pull the
+// 128 logits of the row into registers, release the accumulator, and fold them into a running maximum and
+// two running sums (all visible keys / prompt keys J).  Only tiles that straddle the diagonal are masked
+// and only tiles that reach into J take the prompt-sum path.  Output per head: sum_J / sum_all.
+// ======================================================================================================
+__device__ __forceinline__ float ex2(float x) {          // one MUFU op, flush-to-zero
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct XiTcArgs {
+  const int* n_vis;
+  float* xi_h;
+  uint32_t* status;
+  int cap_in, vis_begin, text_begin, text_end, n_q_heads, group;
+  float scale2;                      // log2(e) / sqrt(dh)
+};
+
+constexpr int XT_STAGES = 2;
+
+template <int DH>
+__global__ void __launch_bounds__(192, 2)
+xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, XiTcArgs a) {
+  constexpr int HALVES = DH / 64;
+  constexpr uint32_t TILE_BYTES = HALVES * 16384;          // 128 rows x DH bf16
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* q_s = base;
+  unsigned char* k_s = base + TILE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + TILE_BYTES * (1 + XT_STAGES));
+  uint64_t* q_full = bars;
+  uint64_t* k_full = bars + 1;                 // [XT_STAGES]
+  uint64_t* k_empty = k_full + XT_STAGES;      // [XT_STAGES]
+  uint64_t* s_full = k_empty + XT_STAGES;      // [2]
+  uint64_t* s_empty = s_full + 2;              // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int qt = gridDim.x - 1 - blockIdx.x;   // longest rows first
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int n = a.n_vis ? min(a.n_vis[b], a.cap_in) : a.cap_in;
+  const int t0 = qt * 128;
+  if (t0 >= n) return;
+  const int nq = min(128, n - t0);
+  const int s_first = a.vis_begin + t0, s_last = s_first + nq - 1;
+  const int nkt = s_last / 128 + 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int i = 0; i < XT_STAGES; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4); }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 256); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tensormap(&q_map);
+      prefetch_tensormap(&k_map);
+      mbar_expect_tx(q_full, TILE_BYTES);
+#pragma unroll
+      for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, s_first, h, b);
+      const int hk = h / a.group;
+      for (int kt = 0; kt < nkt; ++kt) {
+        const int s = kt % XT_STAGES;
+        if (!mbar_wait(&k_empty[s], ((kt / XT_STAGES) & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(&k_full[s], TILE_BYTES);
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf)
+          tma_load_4d(k_s + s * TILE_BYTES + hf * 16384, &k_map, &k_full[s], hf * 64, kt * 128, hk, b);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(128, 128);
+      const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s);
+      bool ok = mbar_wait(q_full, 0, abort_flag);
+      for (int kt = 0; ok && kt < nkt; ++kt) {
+        const int s = kt % XT_STAGES, buf = kt & 1;
+        if (!mbar_wait(&s_empty[buf], ((kt >> 1) & 1) ^ 1, abort_flag)) break;
+        if (!mbar_wait(&k_full[s], (kt / XT_STAGES) & 1, abort_flag)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+          umma_bf16(tmem_base + buf * 128, smem_desc_sw128(q_addr + off),
+                    smem_desc_sw128(k_addr + s * TILE_BYTES + off), idesc, kk > 0);
+        }
+        umma_commit(&k_empty[s]);
+        umma_commit(&s_full[buf]);
+      }
+    }
+  } else {
+    const int quad = warp & 3;                          // TMEM lanes this warp may read
+    const int r = quad * 32 + lane;                     // query row of this thread
+    const uint32_t lane_addr = tmem_base + (uint32_t(quad * 32) << 16);
+    float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
+    const float sc = a.scale2;
+    for (int kt = 0; kt < nkt; ++kt) {
+      const int buf = kt & 1, j0 = kt * 128;
+      if (!mbar_wait(&s_full[buf], (kt >> 1) & 1, abort_flag)) break;
+      tc_fence_after();
+      float v[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(lane_addr + buf * 128 + c * 32, v[c]);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[buf]);
+
+      if (j0 + 127 > s_first) {                         // tile straddles the diagonal: causal mask
+        const int lim = s_first + r - j0;               // last visible column of this row
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c * 32 + i > lim) v[c][i] = -INFINITY;
+      }
+      float mx = v[0][0];
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[c][i]);
+      const float m_new = fmaxf(m_run, mx);
+      const float ms = m_new * sc;
+      float sa = 0.f, st = 0.f;
+      if (j0 < a.text_end && j0 + 128 > a.text_begin) {   // tile reaches into the prompt set J
+        const int lo = a.text_begin - j0, hi = a.text_end - j0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float p = ex2(fmaf(v[c][i], sc, -ms));
+            sa += p;
+            if (c * 32 + i >= lo && c * 32 + i < hi) st += p;
+          }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sa += ex2(fmaf(v[c][i], sc, -ms));
+      }
+      const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
+      l_all = fmaf(l_all, resc, sa);
+      l_txt = fmaf(l_txt, resc, st);
+      m_run = m_new;
+    }
+    if (r < nq && !*abort_flag)
+      a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + t0 + r] = l_txt / l_all;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 256);
+  }
+  if (threadIdx.x == 0 && *abort_flag && a.status) atomicOr(a.status, LIGHTKV_STATUS_TIMEOUT);
+}
+
+bool tc_xi_supported(int head_dim) { return head_dim == 64 || head_dim == 128; }
+
+cudaError_t launch_xi_tc(const LayerLaunch& L) {
+  const lightkv_layer_args_t* a = L.a;
+  const int rows = a->seq_rows > 0 ? a->seq_rows : a->vis_begin + L.ws.cap_in + a->n_text_after;
+  CUtensorMap qm, km;
+  if (!make_map_bhnd(&qm, a->q, L.head_dim, rows, L.n_q_heads, L.batch, a->q_row_stride, a->q_head_stride,
+                     a->q_batch_stride, 128) ||
+      !make_map_bhnd(&km, a->k, L.head_dim, rows, L.n_kv_heads, L.batch, a->k_row_stride, a->k_head_stride,
+                     a->k_batch_stride, 128))
+    return cudaErrorInvalidValue;
+  XiTcArgs x;
+  x.n_vis = a->n_vis; x.xi_h = L.ws.xi_h; x.status = a->status; x.cap_in = L.ws.cap_in;
+  x.vis_begin = a->vis_begin; x.text_begin = a->text_begin; x.text_end = a->text_end;
+  x.n_q_heads = L.n_q_heads; x.group = L.n_q_heads / L.n_kv_heads;
+  x.scale2 = 1.4426950408889634f / sqrtf((float)L.head_dim);
+  const dim3 grid((L.ws.cap_in + 127) / 128, L.n_q_heads, L.batch);
+  const size_t smem = size_t(L.head_dim / 64) * 16384 * (1 + XT_STAGES) + 1024 + 256;
+  cudaError_t e;
+  if (L.head_dim == 128) {
+    if ((e = cudaFuncSetAttribute(xi_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    xi_tc_kernel<128><<<grid, 192, smem, L.stream>>>(qm, km, x);
+  } else {
+    if ((e = cudaFuncSetAttribute(xi_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    xi_tc_kernel<64><<<grid, 192, smem, L.stream>>>(qm, km, x);
+  }
+  return cudaGetLastError();
+}
+
+// FD on tensor cores: not built yet, the FMA path is used.
 bool tc_fd_supported(int) { return false; }
-bool tc_xi_supported(int) { return false; }
 cudaError_t launch_fd_tc(const LayerLaunch&) { return cudaErrorNotSupported; }
-cudaError_t launch_xi_tc(const LayerLaunch&) { return cudaErrorNotSupported; }
+
 }  // namespace lkv

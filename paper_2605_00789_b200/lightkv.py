@@ -59,7 +59,7 @@ class _LayerArgs(C.Structure):
                 ("weight", C.c_void_p), ("grp_off", C.c_void_p), ("grp_src", C.c_void_p),
                 ("xi_out", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p),
-                ("trace_events", C.POINTER(C.c_void_p))]
+                ("trace_events", C.POINTER(C.c_void_p)), ("seq_rows", C.c_int32)]
 
 
 TRACE_EVENTS = 6
@@ -223,6 +223,7 @@ def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_beg
     ho = out.hidden_out
     a.hidden_out, a.hidden_out_batch_stride, a.hidden_out_row_stride = ho.data_ptr(), ho.stride(0), ho.stride(1)
     if q is not None:
+        a.seq_rows = q.shape[2]
         a.q, a.q_batch_stride, a.q_head_stride, a.q_row_stride = q.data_ptr(), q.stride(0), q.stride(1), q.stride(2)
     if k is not None:
         a.k, a.k_batch_stride, a.k_head_stride, a.k_row_stride = k.data_ptr(), k.stride(0), k.stride(1), k.stride(2)
