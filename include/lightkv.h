@@ -182,6 +182,27 @@ typedef struct {
  * small), UNSUPPORTED (mode / dtype / engine combination), CUDA (launch failed). */
 int lightkv_compress_layer(const lightkv_plan_t* plan, const lightkv_layer_args_t* args);
 
+/* The paper has no counterpart of this entry point; it exists for deployment only.
+ * Same operation, arguments, outputs and errors as lightkv_compress_layer, for a caller that has no
+ * scratch buffer to give because it may not allocate device memory: code running inside an engine
+ * that handed all of its memory to a pool at start-up, or inside a region where the runtime
+ * forbids allocation.  args->workspace and args->workspace_bytes are ignored; the stage's scratch
+ * is a fixed device array of LIGHTKV_BUILTIN_WS_BYTES that is part of the library image (each GPU
+ * that loads the library keeps that much memory until the process exits).  This function and
+ * everything below it call no cudaMalloc / cudaFree and no allocating library routine.
+ *   - A stage whose lightkv_plan_stage_info().workspace_bytes exceeds LIGHTKV_BUILTIN_WS_BYTES is
+ *     rejected with LIGHTKV_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current) and remembers it; make that first call outside any stream capture.
+ *     LIGHTKV_ERR_CUDA if the lookup fails.
+ *   - All calls on one device share the array, and it keeps what the previous call left.  Nothing
+ *     in it has to start at zero (every kernel of the stage writes what the later ones read), but
+ *     two calls whose kernels overlap on the GPU (different streams, no ordering between them)
+ *     race on it: order such calls, or give all but one of them lightkv_compress_layer with their
+ *     own workspace. */
+#define LIGHTKV_BUILTIN_WS_BYTES (8u << 20)
+int lightkv_compress_layer_builtin_ws(const lightkv_plan_t* plan, const lightkv_layer_args_t* args);
+
 /* Apply a stage's merge map to one layer's K and V (out of place).
  * Contiguous: element (b, h, n, :) of a tensor lives at
  *   base + b*batch_stride + h*head_stride + n*row_stride.

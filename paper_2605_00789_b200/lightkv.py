@@ -81,7 +81,9 @@ class _KvArgs(C.Structure):
 
 
 EXPORTS = ("lightkv_plan", "lightkv_plan_stage_info", "lightkv_plan_destroy", "lightkv_plan_retention",
-           "lightkv_compress_layer", "lightkv_compact_kv", "lightkv_status_string", "lightkv_version")
+           "lightkv_compress_layer", "lightkv_compress_layer_builtin_ws", "lightkv_compact_kv",
+           "lightkv_status_string", "lightkv_version")
+BUILTIN_WS_BYTES = 8 << 20
 
 
 def library_path() -> str:
@@ -106,6 +108,8 @@ def library() -> C.CDLL:
         lib.lightkv_plan_retention.restype = C.c_double
         lib.lightkv_compress_layer.argtypes = [C.c_void_p, C.POINTER(_LayerArgs)]
         lib.lightkv_compress_layer.restype = C.c_int
+        lib.lightkv_compress_layer_builtin_ws.argtypes = [C.c_void_p, C.POINTER(_LayerArgs)]
+        lib.lightkv_compress_layer_builtin_ws.restype = C.c_int
         lib.lightkv_compact_kv.argtypes = [C.c_void_p, C.POINTER(_KvArgs)]
         lib.lightkv_compact_kv.restype = C.c_int
         lib.lightkv_status_string.argtypes = [C.c_int]
@@ -209,12 +213,10 @@ def _stream_handle(stream) -> int:
     return s.cuda_stream
 
 
-def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin: int,
-                   n_text_after: int = 0, text_begin: int = 0, text_end: Optional[int] = None,
-                   q=None, k=None, lse=None, xi=None, n_vis=None, pos=None, stream=None,
-                   trace_events=None) -> None:
-    """lightkv_compress_layer.  hidden [B,N,d]; q [B,H,N,dh]; k [B,H_kv,N,dh] (any strides with a
-    contiguous last dimension); lse [B,H,N] fp32; xi [B,cap_in] fp32; n_vis [B] int32; pos [B,cap_in] int32."""
+def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin: int,
+                n_text_after: int = 0, text_begin: int = 0, text_end: Optional[int] = None,
+                q=None, k=None, lse=None, xi=None, n_vis=None, pos=None, stream=None,
+                trace_events=None) -> _LayerArgs:
     a = _LayerArgs()
     a.struct_size = C.sizeof(_LayerArgs)
     a.stage, a.vis_begin, a.n_text_after = stage, vis_begin, n_text_after
@@ -237,7 +239,25 @@ def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_beg
     if trace_events is not None:      # TRACE_EVENTS torch.cuda.Event objects (enable_timing=True), already created
         assert len(trace_events) == TRACE_EVENTS
         a.trace_events = (C.c_void_p * TRACE_EVENTS)(*[e.cuda_event for e in trace_events])
+    return a
+
+
+def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, **kw) -> None:
+    """lightkv_compress_layer.  hidden [B,N,d]; keywords: vis_begin, n_text_after, text_begin, text_end,
+    q [B,H,N,dh], k [B,H_kv,N,dh] (any strides with a contiguous last dimension), lse [B,H,N] fp32,
+    xi [B,cap_in] fp32, n_vis [B] int32, pos [B,cap_in] int32, stream, trace_events."""
+    a = _layer_args(plan, stage, hidden, out, **kw)
     _check(library().lightkv_compress_layer(plan.handle, C.byref(a)), "lightkv_compress_layer")
+
+
+def compress_layer_builtin_ws(plan: Plan, stage: int, hidden, out: StageBuffers, **kw) -> None:
+    """lightkv_compress_layer_builtin_ws: same call, but the stage's scratch is the fixed array inside
+    the library (BUILTIN_WS_BYTES), so the workspace tensor of `out` is not used.  Meant for callers
+    that may not allocate device memory; stages needing more scratch than that are refused."""
+    a = _layer_args(plan, stage, hidden, out, **kw)
+    a.workspace, a.workspace_bytes = None, 0
+    _check(library().lightkv_compress_layer_builtin_ws(plan.handle, C.byref(a)),
+           "lightkv_compress_layer_builtin_ws")
 
 
 def compact_kv(plan: Plan, stage: int, out: StageBuffers, k_src, v_src, k_dst, v_dst, *, vis_begin: int,

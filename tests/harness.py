@@ -77,8 +77,9 @@ def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_t
 
 
 def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0, text_range=None,
-              lse=None, kv_mode="merge", paged=0, device="cuda"):
-    """Run lightkv_compress_layer + lightkv_compact_kv on the device; returns numpy outputs."""
+              lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None):
+    """Run lightkv_compress_layer (or `layer_fn`, a binding function with the same signature) +
+    lightkv_compact_kv on the device; returns numpy outputs."""
     import torch
     import paper_2605_00789_b200 as L
     info = plan.stage_info(stage)
@@ -101,9 +102,9 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
     n_seq_out = vb + info.cap_out + n_text_after
     out = L.StageBuffers(plan, stage, n_seq_out, device)
     out.hidden_out.fill_(float("nan"))
-    L.compress_layer(plan, stage, hidden, out, vis_begin=vb, n_text_after=n_text_after, text_begin=tb,
-                     text_end=te, n_vis=torch.from_numpy(inp["n_vis"]).to(device),
-                     pos=torch.from_numpy(pos).to(device), **kw)
+    (layer_fn or L.compress_layer)(plan, stage, hidden, out, vis_begin=vb, n_text_after=n_text_after,
+                                   text_begin=tb, text_end=te, n_vis=torch.from_numpy(inp["n_vis"]).to(device),
+                                   pos=torch.from_numpy(pos).to(device), **kw)
     res = {"out": out}
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     if "k" in inp and "v" in inp:

@@ -147,6 +147,25 @@ def test_calls_reject_bad_arguments_before_any_launch(L):
     assert lib.lightkv_plan_retention(None) < 0
 
 
+def test_builtin_workspace_entry_rejects_oversized_stages_on_the_host(L):
+    lib = L.library()
+    a = L.lightkv._LayerArgs()
+    p = _plan(L)
+    assert lib.lightkv_compress_layer_builtin_ws(p.handle, C.byref(a)) == -1     # struct_size
+    assert lib.lightkv_compress_layer_builtin_ws(None, C.byref(a)) == -1
+    a.struct_size = C.sizeof(a)
+    a.stage = 7
+    assert lib.lightkv_compress_layer_builtin_ws(p.handle, C.byref(a)) == -1     # stage
+    # 64 samples x 32 heads x 2880 tokens of per-head xi alone exceed the built-in array
+    big = _plan(L, batch=64, hidden=4096, n_q_heads=32, n_kv_heads=32, head_dim=128, n_layers=32,
+                tiles=[(24, 24)] * 5, layers=[12], windows=[6], keep=[0.5], max_text=128)
+    assert big.stage_info(0).workspace_bytes > L.BUILTIN_WS_BYTES
+    a.stage = 0
+    assert lib.lightkv_compress_layer_builtin_ws(big.handle, C.byref(a)) == -3   # before any CUDA call
+    header = open(os.path.join(ROOT, "include", "lightkv.h")).read()
+    assert re.search(r"#define LIGHTKV_BUILTIN_WS_BYTES \(8u << 20\)", header) and L.BUILTIN_WS_BYTES == 8 << 20
+
+
 def test_missing_library_fails_loudly(L, monkeypatch):
     from paper_2605_00789_b200 import lightkv
     monkeypatch.setattr(lightkv, "_LIB", None)
