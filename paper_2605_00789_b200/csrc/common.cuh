@@ -9,6 +9,7 @@
 namespace lkv {
 
 constexpr int kMaxTiles = 32;          // image tiles / frames per sample
+constexpr int kFdTile = 128;           // A (and B) entries per tile of the tensor-core FD kernel
 constexpr int kMaxWindows = 2048;      // windows per sample (window-build kernel keeps 32 x n_windows u16 counters in smem)
 
 // Grid geometry of one stage, passed by value to the kernels.
@@ -21,6 +22,15 @@ struct Geometry {
   int cols[kMaxTiles];
 };
 
+// Tiling of one sample's A x B pairs for the tensor-core FD kernel.  Consecutive groups of `wpt`
+// windows share one tile while every window has at most 128 A entries; larger windows are cut into
+// blocks_a x blocks_b blocks of 128 x 128 entries (wpt = 1).
+struct FdTiling {
+  int n_tiles;                         // groups * blocks_a * blocks_b
+  int wpt;                             // windows per group
+  int blocks_a, blocks_b;
+};
+
 // Per-stage views into the caller's workspace (all DEVICE pointers, per-sample row strides in elements).
 struct Workspace {
   int* win_off;    // [B, n_windows + 1]  first window-sorted slot of each window
@@ -30,8 +40,9 @@ struct Workspace {
   int* a_tok;      // [B, cap_a]          token index of each A entry (entries grouped by window)
   int* a_win;      // [B, cap_a]          window of each A entry
   int* b_tok;      // [B, cap_b]          token index of each B entry
-  float* a_f;      // [B, cap_a]          lowest FD of each A entry
-  int* a_best;     // [B, cap_a]          token index of its best B node
+  unsigned long long* a_key;  // [B, cap_a]  (orderable(lowest FD) << 32) | B entry index of the best partner;
+                              //             all ones while no partner is known (set by the window build)
+  FdTiling* fd_tiling;        // [B]         how the tensor-core FD kernel cuts this sample into tiles
   float* xi_h;     // [B, H, cap_in]      per-head attention mass on the prompt (ATTN modes)
   float* xi;       // [B, cap_in]
   int* partner;    // [B, cap_in]         token an A token is merged into, -1 = survives

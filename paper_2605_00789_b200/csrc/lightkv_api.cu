@@ -17,6 +17,7 @@ struct StagePlan {
   bool exact;      // cap_in is the exact count (schedule so far is data independent)
   bool exact_out;  // cap_out too
   bool use_tc;
+  int fd_tiles;    // upper bound on the tiles per sample of the tensor-core FD kernel
   Geometry geo;
   size_t ws_bytes;
   size_t off[13];     // byte offsets of the Workspace arrays
@@ -35,12 +36,23 @@ namespace lkv {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Tiles per sample the window-build kernel will report when the largest window has max_a A entries
+// and max_b B entries (same rule as the kernel; non-decreasing in both).
+static int fd_tile_count(int n_windows, int max_a, int max_b) {
+  if (max_b <= 0) return 0;
+  if (max_a <= kFdTile) {
+    const int wpt = std::min(kFdTile / std::max(max_a, 1), n_windows);
+    return (n_windows + wpt - 1) / wpt;
+  }
+  return n_windows * ((max_a + kFdTile - 1) / kFdTile) * ((max_b + kFdTile - 1) / kFdTile);
+}
+
 static void layout_workspace(const lightkv_plan_t& p, StagePlan& s) {
   const size_t B = p.cfg.batch, nW1 = s.n_windows + 1;
   const bool attn = p.cfg.xi_mode == LIGHTKV_XI_ATTN_FULL || p.cfg.xi_mode == LIGHTKV_XI_ATTN_LSE;
   const size_t sizes[13] = {
       B * nW1 * 4, B * nW1 * 4, B * s.cap_in * 4, B * s.cap_in * 4, B * s.cap_a * 4, B * s.cap_a * 4,
-      B * s.cap_b * 4, B * s.cap_a * 4, B * s.cap_a * 4,
+      B * s.cap_b * 4, B * s.cap_a * 8, B * sizeof(FdTiling),
       attn ? B * p.cfg.n_q_heads * s.cap_in * 4 : 0, B * s.cap_in * 4, B * s.cap_in * 4, B * s.cap_in * 4};
   size_t off = 0;
   for (int i = 0; i < 13; ++i) { s.off[i] = off; off += align_up(sizes[i], 256); }
@@ -57,8 +69,8 @@ static Workspace bind_workspace(const StagePlan& s, void* base) {
   w.a_tok = reinterpret_cast<int*>(p + s.off[4]);
   w.a_win = reinterpret_cast<int*>(p + s.off[5]);
   w.b_tok = reinterpret_cast<int*>(p + s.off[6]);
-  w.a_f = reinterpret_cast<float*>(p + s.off[7]);
-  w.a_best = reinterpret_cast<int*>(p + s.off[8]);
+  w.a_key = reinterpret_cast<unsigned long long*>(p + s.off[7]);
+  w.fd_tiling = reinterpret_cast<FdTiling*>(p + s.off[8]);
   w.xi_h = reinterpret_cast<float*>(p + s.off[9]);
   w.xi = reinterpret_cast<float*>(p + s.off[10]);
   w.partner = reinterpret_cast<int*>(p + s.off[11]);
@@ -167,6 +179,14 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
       sp.cap_a = (sp.cap_in + sp.n_windows) / 2;
       sp.cap_b = sp.cap_in / 2;
     }
+    {  // Whatever positions the caller passes, a window holds at most the tokens of its grid cell
+       // (balanced cells: ceil(rows/w) x ceil(cols/w)); the tile count is non-decreasing in that size.
+      int cell = 0;
+      for (int t = 0; t < c->n_tiles; ++t)
+        cell = std::max(cell, ((g.rows[t] + sp.w - 1) / sp.w) * ((g.cols[t] + sp.w - 1) / sp.w));
+      const int max_a = (std::min(cell, sp.cap_in) + 1) / 2;
+      sp.fd_tiles = fd_tile_count(g.n_windows, max_a, max_a);
+    }
     if (!exact) {   // data-dependent from here on: every window keeps at most ceil(keep n_w) tokens
       long long bound = (long long)ceil(sp.keep * sp.cap_in) + sp.n_windows;
       sp.cap_out = (int)std::min<long long>(bound, sp.cap_in);
@@ -248,6 +268,7 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
   LayerLaunch L;
   L.batch = c.batch; L.hidden = c.hidden; L.n_q_heads = c.n_q_heads; L.n_kv_heads = c.n_kv_heads;
   L.head_dim = c.head_dim; L.dtype = c.dtype; L.xi_mode = c.xi_mode; L.keep = s.keep; L.geo = s.geo;
+  L.fd_tiles = s.fd_tiles;
   L.ws = bind_workspace(s, a->workspace); L.a = a; L.stream = static_cast<cudaStream_t>(a->stream);
 
   cudaEvent_t* ev = reinterpret_cast<cudaEvent_t*>(a->trace_events);

@@ -1,5 +1,7 @@
 // liblightkv kernels, part 1: window build, fp32-FMA contractions (FD, xi), selection + merge map,
 // weighted merge of hidden states, K/V merge-compaction.  sm_100a.
+#include <algorithm>
+
 #include "launch.h"
 
 namespace lkv {
@@ -35,6 +37,8 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
   int* a_tok = ws.a_tok + size_t(b) * ws.cap_a;
   int* a_win = ws.a_win + size_t(b) * ws.cap_a;
   int* b_tok = ws.b_tok + size_t(b) * ws.cap_b;
+  unsigned long long* a_key = ws.a_key + size_t(b) * ws.cap_a;
+  __shared__ int max_ab[2][32];
 
   for (int i = tid; i < 32 * nW; i += blockDim.x) cnt[i] = 0;
   __syncthreads();
@@ -96,6 +100,34 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
     ws.win_off[size_t(b) * (nW + 1) + w] = wsum[w];
     ws.a_off[size_t(b) * (nW + 1) + w] = asum[w];
   }
+  {  // largest A and B side of any window -> tiling of the tensor-core FD kernel
+    int ma = 0, mb = 0;
+    for (int w = tid; w < nW; w += blockDim.x) {
+      const int na = asum[w + 1] - asum[w];
+      ma = max(ma, na);
+      mb = max(mb, wsum[w + 1] - wsum[w] - na);
+    }
+    ma = __reduce_max_sync(0xffffffffu, ma);
+    mb = __reduce_max_sync(0xffffffffu, mb);
+    if (lane == 0) { max_ab[0][wp] = ma; max_ab[1][wp] = mb; }
+    __syncthreads();
+    if (wp == 0) {
+      ma = __reduce_max_sync(0xffffffffu, max_ab[0][lane]);
+      mb = __reduce_max_sync(0xffffffffu, max_ab[1][lane]);
+      if (lane == 0) {
+        FdTiling t;
+        if (ma <= kFdTile) {
+          t.wpt = ma > 0 ? min(kFdTile / ma, nW) : nW;
+          t.blocks_a = 1; t.blocks_b = 1;
+        } else {
+          t.wpt = 1;
+          t.blocks_a = (ma + kFdTile - 1) / kFdTile; t.blocks_b = (mb + kFdTile - 1) / kFdTile;
+        }
+        t.n_tiles = (mb > 0) ? ((nW + t.wpt - 1) / t.wpt) * t.blocks_a * t.blocks_b : 0;
+        ws.fd_tiling[b] = t;
+      }
+    }
+  }
 
   // pass B: local rank, A / B entry lists
   for (int base = s0; base < s1; base += 32) {
@@ -116,7 +148,7 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
         if (e < ws.cap_b) b_tok[e] = i;
       } else {
         const int e = asum[w] + (l >> 1);
-        if (e < ws.cap_a) { a_tok[e] = i; a_win[e] = w; }
+        if (e < ws.cap_a) { a_tok[e] = i; a_win[e] = w; a_key[e] = ~0ull; }
       }
     }
     __syncwarp();
@@ -194,7 +226,7 @@ fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_s
 
   const int tx = tid & 15, ty = tid >> 4;            // 4 B columns x 2 A rows per thread
   float best_f = 3.0e38f;                            // threads < ne: running minimum of their A row
-  int best_tok = -1;
+  int best_e = -1;                                   // ... and the B entry that attains it
   float ssa = 0.f;                                   // threads < FD_TA: squared norm of A row tid
 
   for (int cb = bb0; cb < bb1; cb += FD_TB) {
@@ -252,15 +284,13 @@ fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_s
         const float den = na * sqrtf(b_ss[e - cb]);
         const float cosv = den > 0.f ? Gs[tid][e - cb] / den : 0.f;
         const float fd = 1.0f - cosv;
-        if (fd < best_f) { best_f = fd; best_tok = b_row[e - cb]; }
+        if (fd < best_f) { best_f = fd; best_e = e; }
       }
     }
     __syncthreads();
   }
-  if (tid < ne) {
-    ws.a_f[size_t(b) * ws.cap_a + e0 + tid] = best_f;
-    ws.a_best[size_t(b) * ws.cap_a + e0 + tid] = best_tok;
-  }
+  if (tid < ne && best_e >= 0)
+    ws.a_key[size_t(b) * ws.cap_a + e0 + tid] = ((unsigned long long)orderable(best_f) << 32) | (unsigned)best_e;
 }
 
 cudaError_t launch_fd_simt(const LayerLaunch& L) {
@@ -490,8 +520,8 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   const int* tok_l = ws.tok_l + size_t(b) * ws.cap_in;
   const int* a_tok = ws.a_tok + size_t(b) * ws.cap_a;
   const int* a_win = ws.a_win + size_t(b) * ws.cap_a;
-  const float* a_f = ws.a_f + size_t(b) * ws.cap_a;
-  const int* a_best = ws.a_best + size_t(b) * ws.cap_a;
+  const unsigned long long* a_key = ws.a_key + size_t(b) * ws.cap_a;
+  const int* b_tok = ws.b_tok + size_t(b) * ws.cap_b;
   float* xi = ws.xi + size_t(b) * ws.cap_in;
   int* partner = ws.partner + size_t(b) * ws.cap_in;
   int* slot = ws.slot + size_t(b) * ws.cap_in;
@@ -527,15 +557,17 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     if (r <= 0) sel = false;
     else if (r >= e_hi - e_lo) sel = true;
     else {
-      const unsigned long long key = ((unsigned long long)orderable(a_f[e]) << 32) | (unsigned)e;
+      // order by (lowest FD, A entry index): the high word of a_key is the orderable FD
+      const unsigned long long key = (a_key[e] & 0xffffffff00000000ull) | (unsigned)e;
       int rank = 0;
       for (int e2 = e_lo; e2 < e_hi; ++e2) {
-        const unsigned long long k2 = ((unsigned long long)orderable(a_f[e2]) << 32) | (unsigned)e2;
+        const unsigned long long k2 = (a_key[e2] & 0xffffffff00000000ull) | (unsigned)e2;
         rank += (k2 < key);
       }
       sel = rank < r;
     }
-    if (sel && a_best[e] >= 0) partner[a_tok[e]] = a_best[e];
+    const unsigned best_e = (unsigned)(a_key[e] & 0xffffffffu);
+    if (sel && best_e != 0xffffffffu) partner[a_tok[e]] = b_tok[best_e];
   }
   __syncthreads();
 
@@ -703,8 +735,12 @@ cudaError_t launch_merge_rows(const LayerLaunch& L) {
 
 // =====================================================================================================
 // K/V merge-compaction ("key and value tokens are compressed simultaneously for later layers").
-// One CTA per output token; its threads cover (K|V, head, 16-byte chunk).  The stage's merge map is
-// applied per KV head; contiguous (strided) or paged (block-table) addressing on either side.
+// The stage's merge map is applied per KV head; contiguous (strided) or paged (block-table) addressing
+// on either side.  A CTA takes a few consecutive output tokens (as many as give its threads four
+// 16-byte units each).  It first resolves, once per token, where the token goes and which source
+// tokens feed it with which weight (shared memory), then every thread issues the loads of all its
+// units back to back before it touches any of them, so that each thread keeps up to eight 16-byte
+// loads in flight.  Groups of one are copied; larger groups are summed in fp32 in member order.
 // =====================================================================================================
 struct KvAddr {
   int64_t batch_stride, head_stride, row_stride, page_stride;
@@ -717,55 +753,105 @@ struct KvAddr {
   }
 };
 
+constexpr int KV_THREADS = 256, KV_ITEMS = 4, KV_MAXM = 8, KV_MAXROWS = 8;
+
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(KV_THREADS)
 kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* __restrict__ k_dst,
                   T* __restrict__ v_dst, KvAddr sa, KvAddr da, int n_kv_heads, int dh, int vis_begin,
-                  int n_text_after, int cap_in, int cap_out, int gather,
+                  int n_text_after, int cap_in, int cap_out, int gather, int rows_per_cta,
                   const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
                   const int* __restrict__ grp_off, const int* __restrict__ grp_src,
                   const float* __restrict__ weight) {
   constexpr int V = Vec<T>::n;
-  const int b = blockIdx.y, row = blockIdx.x;
+  __shared__ int64_t s_src[KV_MAXROWS][KV_MAXM];     // element offset of each member's token
+  __shared__ float s_w[KV_MAXROWS][KV_MAXM];
+  __shared__ int64_t s_dst[KV_MAXROWS];
+  __shared__ int s_cnt[KV_MAXROWS], s_g0[KV_MAXROWS];
+
+  const int b = blockIdx.y, row0 = blockIdx.x * rows_per_cta, tid = threadIdx.x;
   const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
   const int n_out = n_vis_out[b];
-  if (row >= vis_begin + n_out + n_text_after) return;
-  const int ch = dh / V, per_kv = n_kv_heads * ch, units = 2 * per_kv;
-  const int64_t d_tok = da.token(b, row);
-  const bool text = row < vis_begin || row >= vis_begin + n_out;
-  int g0 = 0, g1 = 1;
-  int64_t s_tok = 0;
+  const int total_rows = vis_begin + n_out + n_text_after;
+  if (row0 >= total_rows) return;
   const int* gs = grp_src + size_t(b) * cap_in;
   const float* wt = weight + size_t(b) * cap_in;
-  if (text) {
-    s_tok = sa.token(b, row < vis_begin ? row : row - n_out + n_in);
-  } else {
-    const int* go = grp_off + size_t(b) * (cap_out + 1);
-    g0 = go[row - vis_begin];
-    g1 = gather ? g0 + 1 : go[row - vis_begin + 1];
-    if (g1 - g0 == 1) s_tok = sa.token(b, vis_begin + gs[g0]);
+  const int* go = grp_off + size_t(b) * (cap_out + 1);
+
+  if (tid < rows_per_cta * KV_MAXM) {
+    const int r = tid / KV_MAXM, m = tid - r * KV_MAXM, row = row0 + r;
+    int cnt = 0;
+    if (row < total_rows) {
+      if (row < vis_begin || row >= vis_begin + n_out) {          // text row: copied
+        cnt = 1;
+        if (m == 0) {
+          s_src[r][0] = sa.token(b, row < vis_begin ? row : row - n_out + n_in);
+          s_w[r][0] = 1.0f;
+          s_g0[r] = 0;
+        }
+      } else {
+        const int g0 = go[row - vis_begin];
+        cnt = gather ? 1 : go[row - vis_begin + 1] - g0;
+        if (m < cnt) {
+          const int i = gs[g0 + m];
+          s_src[r][m] = sa.token(b, vis_begin + i);
+          s_w[r][m] = wt[i];
+        }
+        if (m == 0) s_g0[r] = g0;
+      }
+      if (m == 0) s_dst[r] = da.token(b, row);
+    }
+    if (m == 0) s_cnt[r] = cnt;
   }
-  for (int u = threadIdx.x; u < units; u += blockDim.x) {
-    const int kv = u / per_kv, rem = u - kv * per_kv, h = rem / ch, c = rem - h * ch;
-    const T* s = kv ? v_src : k_src;
-    T* dp = (kv ? v_dst : k_dst) + d_tok + int64_t(h) * da.head_stride + c * V;
-    const int64_t inner = int64_t(h) * sa.head_stride + c * V;
-    if (text || g1 - g0 == 1) {                        // copy (weight of a lone survivor is exactly 1)
-      st_stream16(dp, ld_stream16(s + s_tok + inner));
-      continue;
-    }
-    float acc[V];
+  __syncthreads();
+
+  const int ch = dh / V, per_kv = n_kv_heads * ch, units = 2 * per_kv;
+  const int total_items = rows_per_cta * units;
+  for (int base = 0; base < total_items; base += KV_THREADS * KV_ITEMS) {
+    uint4 v[KV_ITEMS][2];
+    int cnt[KV_ITEMS], rr[KV_ITEMS];
+    const T* sp[KV_ITEMS];
+    T* dp[KV_ITEMS];
 #pragma unroll
-    for (int j = 0; j < V; ++j) acc[j] = 0.f;
-    for (int g = g0; g < g1; ++g) {
-      const int i = gs[g];
-      const float wv = wt[i];
-      float f[V];
-      unpack16(ld_stream16(s + sa.token(b, vis_begin + i) + inner), f, T());
-#pragma unroll
-      for (int j = 0; j < V; ++j) acc[j] = fmaf(wv, f[j], acc[j]);
+    for (int j = 0; j < KV_ITEMS; ++j) {
+      const int idx = base + j * KV_THREADS + tid;
+      cnt[j] = 0;
+      if (idx >= total_items) continue;
+      const int r = idx / units, u = idx - r * units;
+      const int kv = u / per_kv, rem = u - kv * per_kv, h = rem / ch, c = rem - h * ch;
+      rr[j] = r;
+      cnt[j] = s_cnt[r];
+      if (cnt[j] == 0) continue;
+      sp[j] = (kv ? v_src : k_src) + int64_t(h) * sa.head_stride + c * V;
+      dp[j] = (kv ? v_dst : k_dst) + s_dst[r] + int64_t(h) * da.head_stride + c * V;
+      v[j][0] = ld_stream16(sp[j] + s_src[r][0]);
+      if (cnt[j] > 1) v[j][1] = ld_stream16(sp[j] + s_src[r][1]);
     }
-    st_stream16(dp, pack16(acc, T()));
+#pragma unroll
+    for (int j = 0; j < KV_ITEMS; ++j) {
+      if (cnt[j] == 0) continue;
+      if (cnt[j] == 1) { st_stream16(dp[j], v[j][0]); continue; }   // lone survivor / text / gather: copy
+      const int r = rr[j];
+      float acc[V], f[V];
+      unpack16(v[j][0], f, T());
+      const float w0 = s_w[r][0];
+#pragma unroll
+      for (int e = 0; e < V; ++e) acc[e] = w0 * f[e];
+      unpack16(v[j][1], f, T());
+      const float w1 = s_w[r][1];
+#pragma unroll
+      for (int e = 0; e < V; ++e) acc[e] = fmaf(w1, f[e], acc[e]);
+      for (int m = 2; m < cnt[j]; ++m) {
+        int64_t off;
+        float wv;
+        if (m < KV_MAXM) { off = s_src[r][m]; wv = s_w[r][m]; }
+        else { const int i = gs[s_g0[r] + m]; off = sa.token(b, vis_begin + i); wv = wt[i]; }
+        unpack16(ld_stream16(sp[j] + off), f, T());
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = fmaf(wv, f[e], acc[e]);
+      }
+      st_stream16(dp[j], pack16(acc, T()));
+    }
   }
 }
 
@@ -775,20 +861,23 @@ cudaError_t launch_kv_compact(const KvLaunch& K) {
             a->page_size > 0 ? a->src_block_table : nullptr, a->page_size, a->max_blocks};
   KvAddr da{a->dst_batch_stride, a->dst_head_stride, a->dst_row_stride, a->dst_page_stride,
             a->page_size > 0 ? a->dst_block_table : nullptr, a->page_size, a->max_blocks};
-  const dim3 grid(a->vis_begin + K.cap_out + a->n_text_after, K.batch);
+  const int units = 2 * K.n_kv_heads * (K.head_dim * (K.dtype == LIGHTKV_BF16 ? 2 : 4) / 16);
+  const int rows_per_cta = std::max(1, std::min(KV_MAXROWS, KV_THREADS * KV_ITEMS / units));
+  const int rows = a->vis_begin + K.cap_out + a->n_text_after;
+  const dim3 grid((rows + rows_per_cta - 1) / rows_per_cta, K.batch);
   const int gather = a->mode == LIGHTKV_KV_GATHER;
   if (K.dtype == LIGHTKV_BF16)
-    kv_compact_kernel<__nv_bfloat16><<<grid, 256, 0, K.stream>>>(
+    kv_compact_kernel<__nv_bfloat16><<<grid, KV_THREADS, 0, K.stream>>>(
         static_cast<const __nv_bfloat16*>(a->k_src), static_cast<const __nv_bfloat16*>(a->v_src),
         static_cast<__nv_bfloat16*>(a->k_dst), static_cast<__nv_bfloat16*>(a->v_dst), sa, da, K.n_kv_heads,
-        K.head_dim, a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, a->n_vis, a->n_vis_out,
-        a->grp_off, a->grp_src, a->weight);
+        K.head_dim, a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, rows_per_cta, a->n_vis,
+        a->n_vis_out, a->grp_off, a->grp_src, a->weight);
   else
-    kv_compact_kernel<float><<<grid, 256, 0, K.stream>>>(
+    kv_compact_kernel<float><<<grid, KV_THREADS, 0, K.stream>>>(
         static_cast<const float*>(a->k_src), static_cast<const float*>(a->v_src),
         static_cast<float*>(a->k_dst), static_cast<float*>(a->v_dst), sa, da, K.n_kv_heads, K.head_dim,
-        a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, a->n_vis, a->n_vis_out, a->grp_off,
-        a->grp_src, a->weight);
+        a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, rows_per_cta, a->n_vis, a->n_vis_out,
+        a->grp_off, a->grp_src, a->weight);
   return cudaGetLastError();
 }
 

@@ -156,7 +156,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     const float sc = a.scale2;
     for (int kt = 0; kt < nkt; ++kt) {
       const int buf = kt & 1, j0 = kt * 128;
-      if (!mbar_wait(&s_full[buf], (kt >> 1) & 1, abort_flag)) break;
+      const bool landed = mbar_wait(&s_full[buf], (kt >> 1) & 1, abort_flag);
+      if (!__all_sync(0xffffffffu, landed)) break;        // the TMEM loads below are warp-wide
       tc_fence_after();
       float v[4][32];
 #pragma unroll
@@ -244,8 +245,237 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   return cudaGetLastError();
 }
 
-// FD on tensor cores: not built yet, the FMA path is used.
-bool tc_fd_supported(int) { return false; }
-cudaError_t launch_fd_tc(const LayerLaunch&) { return cudaErrorNotSupported; }
+// ======================================================================================================
+// FD + best partner on tensor cores (Eq. "similarity", Step 2).
+//
+// One CTA per tile of up to 128 A entries x 128 B entries (see FdTiling): a group of whole windows, or
+// one 128 x 128 block of a large window.  The rows of a tile are scattered over the sequence (they are
+// listed by a_tok / b_tok), so eight warps gather them with 16-byte cp.async copies, eight threads per
+// 128-byte row segment, straight into the 128-byte-swizzled K-major layout tcgen05 reads, through a
+// 3-stage ring of 64-column chunks.  Each thread re-reads the 16-byte pieces it fetched to accumulate
+// the rows' squared norms, so X is read from HBM exactly once.  A ninth warp issues
+// G += X_A X_B^T (128 x 128 x 64 per chunk, bf16 -> fp32 in TMEM).  After the last chunk the loader
+// warps turn into the epilogue: one thread per A row scans the FD of the columns that belong to the
+// row's own window and keeps the minimum (ties: lowest B index).  Blocks of a large window combine
+// through a 64-bit atomicMin on (orderable FD, B index), which is order independent.
+// ======================================================================================================
+struct FdTcArgs {
+  const __nv_bfloat16* x;              // first vision row of sample 0
+  int64_t batch_stride, row_stride;    // elements
+  int d;
+  Workspace ws;
+  uint32_t* status;
+};
+
+constexpr int FT_STAGES = 3;
+constexpr int FT_LOADERS = 256;
+constexpr uint32_t FT_OPERAND_BYTES = kFdTile * 128;      // 128 rows x 64 bf16
+constexpr uint32_t FT_STAGE_BYTES = 2 * FT_OPERAND_BYTES;
+constexpr size_t FT_SMEM = size_t(FT_STAGES) * FT_STAGE_BYTES + 1024 /* alignment */ + 128 /* barriers */ +
+                           4 * kFdTile * sizeof(float);
+
+__global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + FT_STAGES * FT_STAGE_BYTES);
+  uint64_t* full = bars;                        // [FT_STAGES] chunk landed (all loader threads arrive)
+  uint64_t* empty = full + FT_STAGES;           // [FT_STAGES] chunk consumed (MMA commit)
+  uint64_t* acc_full = empty + FT_STAGES;       // accumulator complete
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* a_nrm = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(bars) + 128);   // [128]
+  float* b_nrm = a_nrm + kFdTile;                                                          // [128]
+  float* red_f = b_nrm + kFdTile;                                                          // [128]
+  int* red_c = reinterpret_cast<int*>(red_f + kFdTile);                                    // [128]
+
+  const int b = blockIdx.y, tile = blockIdx.x;
+  const FdTiling tl = a.ws.fd_tiling[b];
+  if (tile >= tl.n_tiles) return;
+  const int nW = a.ws.n_windows;
+  const int* win_off = a.ws.win_off + size_t(b) * (nW + 1);
+  const int* a_off = a.ws.a_off + size_t(b) * (nW + 1);
+  const int per_group = tl.blocks_a * tl.blocks_b;
+  const int grp = tile / per_group, rem = tile - grp * per_group;
+  const int ia = rem / tl.blocks_b, ib = rem - ia * tl.blocks_b;
+  const int w0 = min(grp * tl.wpt, nW), w1 = min(nW, w0 + tl.wpt);
+  const int a0 = a_off[w0] + ia * kFdTile, a1 = min(a_off[w1], a0 + kFdTile);
+  const int b0 = win_off[w0] - a_off[w0] + ib * kFdTile, b1 = min(win_off[w1] - a_off[w1], b0 + kFdTile);
+  if (a0 >= a1 || b0 >= b1) return;             // same for every thread of the CTA
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int i = 0; i < FT_STAGES; ++i) { mbar_init(&full[i], FT_LOADERS); mbar_init(&empty[i], 1); }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 8) { tmem_alloc(tmem_slot, kFdTile); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t stage0 = smem_u32(base);
+  const int nk = (a.d + 63) >> 6;
+
+  if (warp < 8) {
+    // ---- gather: thread = 16-byte piece c of rows g, g+32, g+64, g+96 of the A tile and of the B tile
+    const int c = tid & 7, g = tid >> 3;
+    const unsigned char* xb = reinterpret_cast<const unsigned char*>(a.x + size_t(b) * a.batch_stride);
+    const int* a_tok = a.ws.a_tok + size_t(b) * a.ws.cap_a;
+    const int* b_tok = a.ws.b_tok + size_t(b) * a.ws.cap_b;
+    const unsigned char* ap[4];
+    const unsigned char* bp[4];
+    uint32_t a_ok = 0, b_ok = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int ea = a0 + g + 32 * i, eb = b0 + g + 32 * i;
+      const int ta = ea < a1 ? a_tok[ea] : -1, tb = eb < b1 ? b_tok[eb] : -1;
+      a_ok |= (ta >= 0 ? 1u : 0u) << i;
+      b_ok |= (tb >= 0 ? 1u : 0u) << i;
+      ap[i] = xb + (size_t(max(ta, 0)) * a.row_stride + c * 8) * 2;
+      bp[i] = xb + (size_t(max(tb, 0)) * a.row_stride + c * 8) * 2;
+    }
+    const uint32_t piece = uint32_t(g) * 128 + (uint32_t(c ^ (g & 7)) << 4);   // swizzled offset inside an operand
+    float ssa[4] = {0.f, 0.f, 0.f, 0.f}, ssb[4] = {0.f, 0.f, 0.f, 0.f};
+
+    auto issue = [&](int kc) {
+      const uint32_t sb = stage0 + (kc % FT_STAGES) * FT_STAGE_BYTES + piece;
+      const bool in = kc * 64 + c * 8 < a.d;              // d is a multiple of 8: a piece is all in or all out
+      const size_t koff = in ? size_t(kc) * 128 : 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        cp_async16(sb + i * 4096, ap[i] + koff, (in && ((a_ok >> i) & 1)) ? 16u : 0u);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        cp_async16(sb + FT_OPERAND_BYTES + i * 4096, bp[i] + koff, (in && ((b_ok >> i) & 1)) ? 16u : 0u);
+    };
+    auto sumsq = [](const uint4& v, float acc) {
+      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float lo = __uint_as_float(u[j] << 16), hi = __uint_as_float(u[j] & 0xffff0000u);
+        acc = fmaf(lo, lo, acc);
+        acc = fmaf(hi, hi, acc);
+      }
+      return acc;
+    };
+
+    for (int kc = 0; kc < FT_STAGES - 1; ++kc) {
+      if (kc < nk) issue(kc);
+      cp_async_commit();
+    }
+    bool ok = true;
+    for (int k = 0; k < nk; ++k) {
+      const int kn = k + FT_STAGES - 1;
+      if (kn < nk) {
+        if (!mbar_wait(&empty[kn % FT_STAGES], ((kn / FT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        issue(kn);
+      }
+      cp_async_commit();
+      cp_async_wait<FT_STAGES - 1>();                     // this thread's pieces of chunk k have landed
+      const uint32_t sb = stage0 + (k % FT_STAGES) * FT_STAGE_BYTES + piece;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        ssa[i] = sumsq(ld_shared16(sb + i * 4096), ssa[i]);
+        ssb[i] = sumsq(ld_shared16(sb + FT_OPERAND_BYTES + i * 4096), ssb[i]);
+      }
+      fence_proxy_async();                                // cp.async writes -> visible to the tensor core
+      mbar_arrive(&full[k % FT_STAGES]);
+    }
+    cp_async_wait<0>();
+
+    // ---- norms: the eight threads of a row hold partial sums
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        ssa[i] += __shfl_xor_sync(0xffffffffu, ssa[i], o);
+        ssb[i] += __shfl_xor_sync(0xffffffffu, ssb[i], o);
+      }
+      if (c == 0) { a_nrm[g + 32 * i] = sqrtf(ssa[i]); b_nrm[g + 32 * i] = sqrtf(ssb[i]); }
+    }
+    named_barrier(1, FT_LOADERS);
+
+    // ---- epilogue: thread = A row (TMEM lane); warps 0-3 scan columns 0-63, warps 4-7 columns 64-127
+    ok = ok && mbar_wait(acc_full, 0, abort_flag);
+    ok = __all_sync(0xffffffffu, ok);                     // the TMEM loads below are warp-wide
+    tc_fence_after();
+    const int q = warp & 3, half = warp >> 2, row = q * 32 + lane, e = a0 + row;
+    int lo = 0, hi = 0;
+    if (e < a1) {
+      const int w = a.ws.a_win[size_t(b) * a.ws.cap_a + e];
+      lo = max(win_off[w] - a_off[w], b0) - b0;
+      hi = min(win_off[w + 1] - a_off[w + 1], b1) - b0;
+    }
+    const float na = a_nrm[row];
+    float best = 3.0e38f;
+    int best_c = -1;
+    if (ok) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int c0 = half * 64 + j * 32;
+        float v[32];
+        tmem_ld32(tmem_base + (uint32_t(q * 32) << 16) + c0, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int col = c0 + i;
+          if (col >= lo && col < hi) {
+            const float den = na * b_nrm[col];
+            const float fd = 1.0f - (den > 0.f ? v[i] / den : 0.f);
+            if (fd < best) { best = fd; best_c = col; }
+          }
+        }
+      }
+    }
+    if (half == 1) { red_f[row] = best; red_c[row] = best_c; }
+    named_barrier(1, FT_LOADERS);
+    if (half == 0 && ok && e < a1) {
+      if (red_f[row] < best) { best = red_f[row]; best_c = red_c[row]; }   // ties stay with the lower column
+      if (best_c >= 0) {
+        const unsigned long long key = ((unsigned long long)orderable(best) << 32) | (unsigned)(b0 + best_c);
+        unsigned long long* dst = a.ws.a_key + size_t(b) * a.ws.cap_a + e;
+        if (tl.blocks_b > 1) atomicMin(dst, key); else *dst = key;
+      }
+    }
+  } else if (lane == 0) {
+    // ---- MMA issue
+    constexpr uint32_t idesc = idesc_bf16(kFdTile, kFdTile);
+    for (int k = 0; k < nk; ++k) {
+      const int s = k % FT_STAGES;
+      if (!mbar_wait(&full[s], (k / FT_STAGES) & 1, abort_flag)) break;
+      tc_fence_after();
+      const uint32_t sa = stage0 + s * FT_STAGE_BYTES;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk)
+        umma_bf16(tmem_base, smem_desc_sw128(sa + kk * 32), smem_desc_sw128(sa + FT_OPERAND_BYTES + kk * 32), idesc,
+                  (k | kk) != 0);
+      umma_commit(&empty[s]);
+    }
+    umma_commit(acc_full);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kFdTile);
+  }
+  if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, LIGHTKV_STATUS_TIMEOUT);
+}
+
+bool tc_fd_supported(int hidden) { return hidden % 8 == 0; }
+
+cudaError_t launch_fd_tc(const LayerLaunch& L) {
+  const lightkv_layer_args_t* a = L.a;
+  FdTcArgs f;
+  f.x = static_cast<const __nv_bfloat16*>(a->hidden) + size_t(a->vis_begin) * a->hidden_row_stride;
+  f.batch_stride = a->hidden_batch_stride; f.row_stride = a->hidden_row_stride; f.d = L.hidden;
+  f.ws = L.ws; f.status = a->status;
+  cudaError_t e = cudaFuncSetAttribute(fd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM);
+  if (e != cudaSuccess) return e;
+  if (L.fd_tiles <= 0) return cudaSuccess;
+  fd_tc_kernel<<<dim3(L.fd_tiles, L.batch), FT_LOADERS + 32, FT_SMEM, L.stream>>>(f);
+  return cudaGetLastError();
+}
 
 }  // namespace lkv
