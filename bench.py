@@ -320,13 +320,16 @@ def main():
     value = world * tokens_per_step / (ms_step / 1e3)
 
     ktime = {k: 0.0 for k in KERNELS}       # ms per step, summed over stages
+    kstage = [{k: 0.0 for k in KERNELS} for _ in range(n_stages)]
     for i in range(args.steps):
         for st in range(n_stages):
             e = traces[i][st]
             for j, name in enumerate(L.TRACE_NAMES):
-                ktime[name] += e[j].elapsed_time(e[j + 1])
-            ktime["kv_compact"] += e[-1].elapsed_time(kv_ev[i][st])
-    ktime = {k: v / args.steps for k, v in ktime.items()}
+                kstage[st][name] += e[j].elapsed_time(e[j + 1]) / args.steps
+            kstage[st]["kv_compact"] += e[-1].elapsed_time(kv_ev[i][st]) / args.steps
+    for st in range(n_stages):
+        for k in KERNELS:
+            ktime[k] += kstage[st][k]
     work = algorithmic_work(wl, stages)
     peaks = measured_peaks()
     kernels = {}
@@ -392,7 +395,8 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
                 "us_per_compression_layer": 1e3 * ms_step / n_stages,
-                "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+                "roofline": roofline, "kernels": kernels,
+                "us_by_stage": [{k: round(1e3 * v, 1) for k, v in ks.items()} for ks in kstage], "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                 "gpu_launches": launches_per_step * args.steps,
                 "engine": {st: int(plan.stage_info(st).uses_tensor_cores) for st in range(n_stages)}}
         print(json.dumps(line))

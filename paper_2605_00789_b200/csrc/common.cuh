@@ -24,12 +24,18 @@ struct Geometry {
 
 // Tiling of one sample's A x B pairs for the tensor-core FD kernel.  Consecutive groups of `wpt`
 // windows share one tile while every window has at most 128 A entries; larger windows are cut into
-// blocks_a x blocks_b blocks of 128 x 128 entries (wpt = 1).
+// blocks_a x blocks_b blocks of 128 x 128 entries (wpt = 1).  `passes` * 32 bounds the A (and B)
+// entries of any tile; the kernel sizes its shared-memory stages from it.
 struct FdTiling {
   int n_tiles;                         // groups * blocks_a * blocks_b
   int wpt;                             // windows per group
   int blocks_a, blocks_b;
+  int passes;                          // 1, 2 or 4
+  int pad[3];
 };
+
+// Groups are kept small enough that the whole batch yields about this many tiles (two per SM).
+constexpr int kFdTargetTiles = 296;
 
 // Per-stage views into the caller's workspace (all DEVICE pointers, per-sample row strides in elements).
 struct Workspace {

@@ -36,15 +36,12 @@ namespace lkv {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Tiles per sample the window-build kernel will report when the largest window has max_a A entries
-// and max_b B entries (same rule as the kernel; non-decreasing in both).
-static int fd_tile_count(int n_windows, int max_a, int max_b) {
-  if (max_b <= 0) return 0;
-  if (max_a <= kFdTile) {
-    const int wpt = std::min(kFdTile / std::max(max_a, 1), n_windows);
-    return (n_windows + wpt - 1) / wpt;
-  }
-  return n_windows * ((max_a + kFdTile - 1) / kFdTile) * ((max_b + kFdTile - 1) / kFdTile);
+// Upper bound on the tiles per sample the window-build kernel can report when no window has more than
+// max_a A entries: one tile per window while windows fit a tile, else blocks of 128 x 128 per window.
+static int fd_tile_bound(int n_windows, int max_a) {
+  if (max_a <= kFdTile) return n_windows;
+  const int blocks = (max_a + kFdTile - 1) / kFdTile;
+  return n_windows * blocks * blocks;
 }
 
 static void layout_workspace(const lightkv_plan_t& p, StagePlan& s) {
@@ -180,12 +177,12 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
       sp.cap_b = sp.cap_in / 2;
     }
     {  // Whatever positions the caller passes, a window holds at most the tokens of its grid cell
-       // (balanced cells: ceil(rows/w) x ceil(cols/w)); the tile count is non-decreasing in that size.
+       // (balanced cells: ceil(rows/w) x ceil(cols/w)).
       int cell = 0;
       for (int t = 0; t < c->n_tiles; ++t)
         cell = std::max(cell, ((g.rows[t] + sp.w - 1) / sp.w) * ((g.cols[t] + sp.w - 1) / sp.w));
       const int max_a = (std::min(cell, sp.cap_in) + 1) / 2;
-      sp.fd_tiles = fd_tile_count(g.n_windows, max_a, max_a);
+      sp.fd_tiles = fd_tile_bound(g.n_windows, max_a);
     }
     if (!exact) {   // data-dependent from here on: every window keeps at most ceil(keep n_w) tokens
       long long bound = (long long)ceil(sp.keep * sp.cap_in) + sp.n_windows;

@@ -117,13 +117,19 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
       if (lane == 0) {
         FdTiling t;
         if (ma <= kFdTile) {
-          t.wpt = ma > 0 ? min(kFdTile / ma, nW) : nW;
+          // as few windows per tile as still gives the batch about kFdTargetTiles tiles, at most 128 A entries
+          const int want = (nW * (int)gridDim.x + kFdTargetTiles - 1) / kFdTargetTiles;
+          t.wpt = ma > 0 ? max(1, min(min(kFdTile / ma, nW), want)) : nW;
           t.blocks_a = 1; t.blocks_b = 1;
+          const int rows = t.wpt * ma;
+          t.passes = rows <= 32 ? 1 : (rows <= 64 ? 2 : 4);
         } else {
           t.wpt = 1;
           t.blocks_a = (ma + kFdTile - 1) / kFdTile; t.blocks_b = (mb + kFdTile - 1) / kFdTile;
+          t.passes = 4;
         }
         t.n_tiles = (mb > 0) ? ((nW + t.wpt - 1) / t.wpt) * t.blocks_a * t.blocks_b : 0;
+        t.pad[0] = t.pad[1] = t.pad[2] = 0;
         ws.fd_tiling[b] = t;
       }
     }

@@ -252,12 +252,22 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
 // one 128 x 128 block of a large window.  The rows of a tile are scattered over the sequence (they are
 // listed by a_tok / b_tok), so eight warps gather them with 16-byte cp.async copies, eight threads per
 // 128-byte row segment, straight into the 128-byte-swizzled K-major layout tcgen05 reads, through a
-// 3-stage ring of 64-column chunks.  Each thread re-reads the 16-byte pieces it fetched to accumulate
-// the rows' squared norms, so X is read from HBM exactly once.  A ninth warp issues
-// G += X_A X_B^T (128 x 128 x 64 per chunk, bf16 -> fp32 in TMEM).  After the last chunk the loader
+// ring of three 32 KB stages.  A tile holds at most 32 * passes rows per operand (passes = 1, 2, 4), and
+// a stage holds 4 / passes consecutive 64-column chunks of both operands, so every thread always moves
+// eight 16-byte pieces per stage whatever the tile size, and two stages (64 KB) stay in flight per CTA,
+// two CTAs per SM.  Each thread re-reads the pieces it fetched to accumulate the rows' squared norms,
+// so X is read from HBM exactly once.  A ninth warp issues G += X_A X_B^T (128 x N x 64 per chunk,
+// N = B entries rounded up to 16, bf16 -> fp32 in TMEM).  The MMA always reads 128 A rows (16 KB) from
+// the start of a chunk's A block: rows the tile does not have are never written, overlap other blocks
+// of the same stage, and only feed accumulator rows nobody reads.  After the last chunk the loader
 // warps turn into the epilogue: one thread per A row scans the FD of the columns that belong to the
 // row's own window and keeps the minimum (ties: lowest B index).  Blocks of a large window combine
 // through a 64-bit atomicMin on (orderable FD, B index), which is order independent.
+//
+// Stage layout (offsets in KB), chosen so that the 16 KB A read stays inside the stage:
+//   passes 4: [A 0-16 | B 16-32]                     one chunk
+//   passes 2: [A0 0-8 | B0 8-16 | A1 16-24 | B1 24-32]   two chunks
+//   passes 1: [A0 A1 A2 A3 0-16 | B0 B1 B2 B3 16-32]     four chunks, 4 KB each
 // ======================================================================================================
 struct FdTcArgs {
   const __nv_bfloat16* x;              // first vision row of sample 0
@@ -267,10 +277,9 @@ struct FdTcArgs {
   uint32_t* status;
 };
 
-constexpr int FT_STAGES = 3;
 constexpr int FT_LOADERS = 256;
-constexpr uint32_t FT_OPERAND_BYTES = kFdTile * 128;      // 128 rows x 64 bf16
-constexpr uint32_t FT_STAGE_BYTES = 2 * FT_OPERAND_BYTES;
+constexpr int FT_STAGES = 3;
+constexpr uint32_t FT_STAGE_BYTES = 32 * 1024;
 constexpr size_t FT_SMEM = size_t(FT_STAGES) * FT_STAGE_BYTES + 1024 /* alignment */ + 128 /* barriers */ +
                            4 * kFdTile * sizeof(float);
 
@@ -278,8 +287,8 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + FT_STAGES * FT_STAGE_BYTES);
-  uint64_t* full = bars;                        // [FT_STAGES] chunk landed (all loader threads arrive)
-  uint64_t* empty = full + FT_STAGES;           // [FT_STAGES] chunk consumed (MMA commit)
+  uint64_t* full = bars;                        // [FT_STAGES] stage landed (one arrival per loader warp)
+  uint64_t* empty = full + FT_STAGES;           // [FT_STAGES] stage consumed (MMA commit)
   uint64_t* acc_full = empty + FT_STAGES;       // accumulator complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -298,13 +307,19 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   const int grp = tile / per_group, rem = tile - grp * per_group;
   const int ia = rem / tl.blocks_b, ib = rem - ia * tl.blocks_b;
   const int w0 = min(grp * tl.wpt, nW), w1 = min(nW, w0 + tl.wpt);
-  const int a0 = a_off[w0] + ia * kFdTile, a1 = min(a_off[w1], a0 + kFdTile);
-  const int b0 = win_off[w0] - a_off[w0] + ib * kFdTile, b1 = min(win_off[w1] - a_off[w1], b0 + kFdTile);
+  const int passes = tl.passes;                                      // 1, 2 or 4
+  const int cap_rows = 32 * passes;
+  const int a0 = a_off[w0] + ia * kFdTile, a1 = min(a_off[w1], a0 + cap_rows);
+  const int b0 = win_off[w0] - a_off[w0] + ib * kFdTile, b1 = min(win_off[w1] - a_off[w1], b0 + cap_rows);
   if (a0 >= a1 || b0 >= b1) return;             // same for every thread of the CTA
+  const int n_cols = (b1 - b0 + 15) & ~15;      // MMA N
+  const int kps = 4 / passes;                   // 64-column chunks per stage
+  const int nk = (a.d + 63) >> 6;               // chunks
+  const int nst = (nk + kps - 1) / kps;         // stages' worth of chunks
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int i = 0; i < FT_STAGES; ++i) { mbar_init(&full[i], FT_LOADERS); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < FT_STAGES; ++i) { mbar_init(&full[i], FT_LOADERS / 32); mbar_init(&empty[i], 1); }
     mbar_init(acc_full, 1);
     *abort_flag = 0;
     fence_barrier_init();
@@ -314,40 +329,49 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t stage0 = smem_u32(base);
-  const int nk = (a.d + 63) >> 6;
+  const uint32_t ring = smem_u32(base);
 
   if (warp < 8) {
-    // ---- gather: thread = 16-byte piece c of rows g, g+32, g+64, g+96 of the A tile and of the B tile
+    // ---- gather: thread = 16-byte piece c of rows g + 32 i (i < passes) of both operands, for every chunk
+    //      of the stage; copy t of a stage is (chunk t / passes, row g + 32 (t % passes))
     const int c = tid & 7, g = tid >> 3;
     const unsigned char* xb = reinterpret_cast<const unsigned char*>(a.x + size_t(b) * a.batch_stride);
     const int* a_tok = a.ws.a_tok + size_t(b) * a.ws.cap_a;
     const int* b_tok = a.ws.b_tok + size_t(b) * a.ws.cap_b;
+    const uint32_t piece = uint32_t(g) * 128 + (uint32_t(c ^ (g & 7)) << 4);   // swizzled offset inside a block
     const unsigned char* ap[4];
     const unsigned char* bp[4];
+    uint32_t a_so[4], b_so[4];                            // shared-memory offset of copy t inside a stage
+    int kj[4];                                            // chunk of copy t inside a stage
     uint32_t a_ok = 0, b_ok = 0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int t = 0; t < 4; ++t) {
+      const int i = t & (passes - 1), j = t / passes;
       const int ea = a0 + g + 32 * i, eb = b0 + g + 32 * i;
       const int ta = ea < a1 ? a_tok[ea] : -1, tb = eb < b1 ? b_tok[eb] : -1;
-      a_ok |= (ta >= 0 ? 1u : 0u) << i;
-      b_ok |= (tb >= 0 ? 1u : 0u) << i;
-      ap[i] = xb + (size_t(max(ta, 0)) * a.row_stride + c * 8) * 2;
-      bp[i] = xb + (size_t(max(tb, 0)) * a.row_stride + c * 8) * 2;
+      a_ok |= (ta >= 0 ? 1u : 0u) << t;
+      b_ok |= (tb >= 0 ? 1u : 0u) << t;
+      ap[t] = xb + (size_t(max(ta, 0)) * a.row_stride + c * 8) * 2 + size_t(j) * 128;
+      bp[t] = xb + (size_t(max(tb, 0)) * a.row_stride + c * 8) * 2 + size_t(j) * 128;
+      kj[t] = j;
+      if (passes == 2) { a_so[t] = j * 16384 + i * 4096 + piece; b_so[t] = a_so[t] + 8192; }
+      else { a_so[t] = t * 4096 + piece; b_so[t] = 16384 + t * 4096 + piece; }
     }
-    const uint32_t piece = uint32_t(g) * 128 + (uint32_t(c ^ (g & 7)) << 4);   // swizzled offset inside an operand
     float ssa[4] = {0.f, 0.f, 0.f, 0.f}, ssb[4] = {0.f, 0.f, 0.f, 0.f};
 
-    auto issue = [&](int kc) {
-      const uint32_t sb = stage0 + (kc % FT_STAGES) * FT_STAGE_BYTES + piece;
-      const bool in = kc * 64 + c * 8 < a.d;              // d is a multiple of 8: a piece is all in or all out
-      const size_t koff = in ? size_t(kc) * 128 : 0;
+    // rows the tile does not have and chunks past the hidden size are not fetched at all; the pieces of
+    // the last chunk that lie past the hidden size are zero-filled
+    auto issue = [&](int st, int stage) {
+      const uint32_t sb = ring + stage * FT_STAGE_BYTES;
+      const size_t koff = size_t(st) * kps * 128;
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        cp_async16(sb + i * 4096, ap[i] + koff, (in && ((a_ok >> i) & 1)) ? 16u : 0u);
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        cp_async16(sb + FT_OPERAND_BYTES + i * 4096, bp[i] + koff, (in && ((b_ok >> i) & 1)) ? 16u : 0u);
+      for (int t = 0; t < 4; ++t) {
+        const int kc = st * kps + kj[t];
+        if (kc >= nk) continue;
+        const uint32_t bytes = (kc * 64 + c * 8 < a.d) ? 16u : 0u;   // d is a multiple of 8
+        if ((a_ok >> t) & 1) cp_async16(sb + a_so[t], ap[t] + (bytes ? koff : 0), bytes);
+        if ((b_ok >> t) & 1) cp_async16(sb + b_so[t], bp[t] + (bytes ? koff : 0), bytes);
+      }
     };
     auto sumsq = [](const uint4& v, float acc) {
       const uint32_t u[4] = {v.x, v.y, v.z, v.w};
@@ -360,31 +384,35 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       return acc;
     };
 
-    for (int kc = 0; kc < FT_STAGES - 1; ++kc) {
-      if (kc < nk) issue(kc);
+    for (int st = 0; st < FT_STAGES - 1; ++st) {
+      if (st < nst) issue(st, st);
       cp_async_commit();
     }
     bool ok = true;
-    for (int k = 0; k < nk; ++k) {
-      const int kn = k + FT_STAGES - 1;
-      if (kn < nk) {
-        if (!mbar_wait(&empty[kn % FT_STAGES], ((kn / FT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        issue(kn);
+    for (int st = 0; st < nst; ++st) {
+      const int sn = st + FT_STAGES - 1;
+      if (sn < nst) {
+        if (!mbar_wait(&empty[sn % FT_STAGES], ((sn / FT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        issue(sn, sn % FT_STAGES);
       }
       cp_async_commit();
-      cp_async_wait<FT_STAGES - 1>();                     // this thread's pieces of chunk k have landed
-      const uint32_t sb = stage0 + (k % FT_STAGES) * FT_STAGE_BYTES + piece;
+      cp_async_wait<FT_STAGES - 1>();                     // this thread's pieces of stage st have landed
+      const uint32_t sb = ring + (st % FT_STAGES) * FT_STAGE_BYTES;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        ssa[i] = sumsq(ld_shared16(sb + i * 4096), ssa[i]);
-        ssb[i] = sumsq(ld_shared16(sb + FT_OPERAND_BYTES + i * 4096), ssb[i]);
+      for (int t = 0; t < 4; ++t) {
+        if (st * kps + kj[t] >= nk) continue;
+        if ((a_ok >> t) & 1) ssa[t] = sumsq(ld_shared16(sb + a_so[t]), ssa[t]);
+        if ((b_ok >> t) & 1) ssb[t] = sumsq(ld_shared16(sb + b_so[t]), ssb[t]);
       }
       fence_proxy_async();                                // cp.async writes -> visible to the tensor core
-      mbar_arrive(&full[k % FT_STAGES]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&full[st % FT_STAGES]);
     }
     cp_async_wait<0>();
 
-    // ---- norms: the eight threads of a row hold partial sums
+    // ---- norms: copies of the same row, then the eight threads of a row, hold partial sums
+    if (passes == 2) { ssa[0] += ssa[2]; ssa[1] += ssa[3]; ssb[0] += ssb[2]; ssb[1] += ssb[3]; }
+    if (passes == 1) { ssa[0] += ssa[1] + ssa[2] + ssa[3]; ssb[0] += ssb[1] + ssb[2] + ssb[3]; }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
 #pragma unroll
@@ -392,7 +420,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         ssa[i] += __shfl_xor_sync(0xffffffffu, ssa[i], o);
         ssb[i] += __shfl_xor_sync(0xffffffffu, ssb[i], o);
       }
-      if (c == 0) { a_nrm[g + 32 * i] = sqrtf(ssa[i]); b_nrm[g + 32 * i] = sqrtf(ssb[i]); }
+      if (c == 0 && i < passes) { a_nrm[g + 32 * i] = sqrtf(ssa[i]); b_nrm[g + 32 * i] = sqrtf(ssb[i]); }
     }
     named_barrier(1, FT_LOADERS);
 
@@ -407,13 +435,14 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       lo = max(win_off[w] - a_off[w], b0) - b0;
       hi = min(win_off[w + 1] - a_off[w + 1], b1) - b0;
     }
-    const float na = a_nrm[row];
+    const float na = row < cap_rows ? a_nrm[row] : 0.f;
     float best = 3.0e38f;
     int best_c = -1;
     if (ok) {
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int c0 = half * 64 + j * 32;
+        if (c0 >= n_cols) break;                          // warp-uniform
         float v[32];
         tmem_ld32(tmem_base + (uint32_t(q * 32) << 16) + c0, v);
         tmem_ld_wait();
@@ -440,16 +469,20 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     }
   } else if (lane == 0) {
     // ---- MMA issue
-    constexpr uint32_t idesc = idesc_bf16(kFdTile, kFdTile);
-    for (int k = 0; k < nk; ++k) {
-      const int s = k % FT_STAGES;
-      if (!mbar_wait(&full[s], (k / FT_STAGES) & 1, abort_flag)) break;
+    const uint32_t idesc = idesc_bf16(kFdTile, n_cols);
+    const uint32_t chunk_step = passes == 4 ? 0u : (passes == 2 ? 16384u : 4096u);   // A block to A block
+    const uint32_t b_from_a = passes == 2 ? 8192u : 16384u;
+    for (int st = 0; st < nst; ++st) {
+      const int s = st % FT_STAGES;
+      if (!mbar_wait(&full[s], (st / FT_STAGES) & 1, abort_flag)) break;
       tc_fence_after();
-      const uint32_t sa = stage0 + s * FT_STAGE_BYTES;
+      for (int j = 0; j < kps && st * kps + j < nk; ++j) {
+        const uint32_t sa = ring + s * FT_STAGE_BYTES + j * chunk_step;
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk)
-        umma_bf16(tmem_base, smem_desc_sw128(sa + kk * 32), smem_desc_sw128(sa + FT_OPERAND_BYTES + kk * 32), idesc,
-                  (k | kk) != 0);
+        for (int kk = 0; kk < 4; ++kk)
+          umma_bf16(tmem_base, smem_desc_sw128(sa + kk * 32), smem_desc_sw128(sa + b_from_a + kk * 32), idesc,
+                    (st | j | kk) != 0);
+      }
       umma_commit(&empty[s]);
     }
     umma_commit(acc_full);
