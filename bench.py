@@ -97,12 +97,36 @@ class ClockSampler:
         return out
 
 
+# ------------------------------------------------------------------------------------- multi-rank
+# Samples are independent and the path has no exchange step: rank r compresses its own batch (samples
+# r*batch .. r*batch + batch - 1 of the seeded generator).  The only communication is the timing protocol.
+
+def rank_samples(rank: int, batch: int):
+    return [rank * batch + b for b in range(batch)]
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Slowest rank's value (all-reduce MAX over the default process group); identity for one rank."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(tokens_per_rank_step: int, world: int, ms_step_max: float) -> float:
+    """Units all ranks processed per second, timed by the slowest rank."""
+    return world * tokens_per_rank_step / (ms_step_max / 1e3)
+
+
 # ------------------------------------------------------------------------------------------ workload
 
 def build_inputs(wl, plan, L, torch, device, sample_offset):
     """Generate every stage's inputs on the host (pinned) and upload them.  Stage i+1 is sampled at the
     positions that survive stage i (taken from one untimed run of the library itself)."""
-    samples = [sample_offset + b for b in range(wl.batch)]
+    samples = rank_samples(sample_offset // wl.batch, wl.batch)
     stages, pos = [], None
     for st in range(wl.n_stages):
         info = plan.stage_info(st)
@@ -311,13 +335,9 @@ def main():
     t_end.record()
     barrier()
     clocks = sampler.stop()
-    ms_total = t_begin.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([ms_total], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(t_begin.elapsed_time(t_end), world, device)
     ms_step = ms_total / args.steps
-    value = world * tokens_per_step / (ms_step / 1e3)
+    value = whole_job_throughput(tokens_per_step, world, ms_step)
 
     ktime = {k: 0.0 for k in KERNELS}       # ms per step, summed over stages
     kstage = [{k: 0.0 for k in KERNELS} for _ in range(n_stages)]
@@ -375,12 +395,8 @@ def main():
             e2e_step()
         b.record()
         barrier()
-        ms_e2e = a.elapsed_time(b) / e2e_steps
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": world * tokens_per_step / (ms_e2e / 1e3), "unit": unit, "h2d_bytes_per_step": h2d,
+        ms_e2e = max_over_ranks(a.elapsed_time(b) / e2e_steps, world, device)
+        e2e = {"value": whole_job_throughput(tokens_per_step, world, ms_e2e), "unit": unit, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
 
     cpu = None

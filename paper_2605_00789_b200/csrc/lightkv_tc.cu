@@ -1,4 +1,6 @@
 // liblightkv kernels, part 2: tcgen05 tensor-core contractions fed by TMA (sm_100a).
+#include <algorithm>
+
 #include "launch.h"
 #include "tc_common.cuh"
 
@@ -272,7 +274,7 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
 struct FdTcArgs {
   const __nv_bfloat16* x;              // first vision row of sample 0
   int64_t batch_stride, row_stride;    // elements
-  int d;
+  int d, batch;
   Workspace ws;
   uint32_t* status;
 };
@@ -297,26 +299,6 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   float* red_f = b_nrm + kFdTile;                                                          // [128]
   int* red_c = reinterpret_cast<int*>(red_f + kFdTile);                                    // [128]
 
-  const int b = blockIdx.y, tile = blockIdx.x;
-  const FdTiling tl = a.ws.fd_tiling[b];
-  if (tile >= tl.n_tiles) return;
-  const int nW = a.ws.n_windows;
-  const int* win_off = a.ws.win_off + size_t(b) * (nW + 1);
-  const int* a_off = a.ws.a_off + size_t(b) * (nW + 1);
-  const int per_group = tl.blocks_a * tl.blocks_b;
-  const int grp = tile / per_group, rem = tile - grp * per_group;
-  const int ia = rem / tl.blocks_b, ib = rem - ia * tl.blocks_b;
-  const int w0 = min(grp * tl.wpt, nW), w1 = min(nW, w0 + tl.wpt);
-  const int passes = tl.passes;                                      // 1, 2 or 4
-  const int cap_rows = 32 * passes;
-  const int a0 = a_off[w0] + ia * kFdTile, a1 = min(a_off[w1], a0 + cap_rows);
-  const int b0 = win_off[w0] - a_off[w0] + ib * kFdTile, b1 = min(win_off[w1] - a_off[w1], b0 + cap_rows);
-  if (a0 >= a1 || b0 >= b1) return;             // same for every thread of the CTA
-  const int n_cols = (b1 - b0 + 15) & ~15;      // MMA N
-  const int kps = 4 / passes;                   // 64-column chunks per stage
-  const int nk = (a.d + 63) >> 6;               // chunks
-  const int nst = (nk + kps - 1) / kps;         // stages' worth of chunks
-
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int i = 0; i < FT_STAGES; ++i) { mbar_init(&full[i], FT_LOADERS / 32); mbar_init(&empty[i], 1); }
@@ -330,6 +312,37 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t ring = smem_u32(base);
+  const int nW = a.ws.n_windows;
+  const int nk = (a.d + 63) >> 6;               // 64-column chunks
+
+  // Persistent CTA: work items are the (sample, tile) pairs of the whole batch in sample order; this CTA
+  // takes items blockIdx.x, blockIdx.x + gridDim.x, ...  Barrier phases run on across items: `done` counts
+  // the stage fills this CTA has completed, `n_items` its finished tiles.
+  uint32_t done = 0, n_items = 0;
+  for (int item = blockIdx.x;; item += gridDim.x) {
+  int b = 0, tile = item;
+  while (b < a.batch) {
+    const int nt = a.ws.fd_tiling[b].n_tiles;
+    if (tile < nt) break;
+    tile -= nt;
+    ++b;
+  }
+  if (b >= a.batch) break;                      // same for every thread of the CTA
+  const FdTiling tl = a.ws.fd_tiling[b];
+  const int* win_off = a.ws.win_off + size_t(b) * (nW + 1);
+  const int* a_off = a.ws.a_off + size_t(b) * (nW + 1);
+  const int per_group = tl.blocks_a * tl.blocks_b;
+  const int grp = tile / per_group, rem = tile - grp * per_group;
+  const int ia = rem / tl.blocks_b, ib = rem - ia * tl.blocks_b;
+  const int w0 = min(grp * tl.wpt, nW), w1 = min(nW, w0 + tl.wpt);
+  const int passes = tl.passes;                                      // 1, 2 or 4
+  const int cap_rows = 32 * passes;
+  const int a0 = a_off[w0] + ia * kFdTile, a1 = min(a_off[w1], a0 + cap_rows);
+  const int b0 = win_off[w0] - a_off[w0] + ib * kFdTile, b1 = min(win_off[w1] - a_off[w1], b0 + cap_rows);
+  if (a0 >= a1 || b0 >= b1) continue;           // same for every thread of the CTA
+  const int n_cols = (b1 - b0 + 15) & ~15;      // MMA N
+  const int kps = 4 / passes;                   // chunks per stage
+  const int nst = (nk + kps - 1) / kps;         // stage fills of this tile
 
   if (warp < 8) {
     // ---- gather: thread = 16-byte piece c of rows g + 32 i (i < passes) of both operands, for every chunk
@@ -384,20 +397,28 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       return acc;
     };
 
-    for (int st = 0; st < FT_STAGES - 1; ++st) {
-      if (st < nst) issue(st, st);
-      cp_async_commit();
-    }
+    // fill f of this CTA (counted across tiles) uses stage f % 3; it may be written once the MMAs of fill
+    // f - 3 have completed, and is complete for the MMA warp on phase (f / 3) & 1 of full[]
     bool ok = true;
-    for (int st = 0; st < nst; ++st) {
-      const int sn = st + FT_STAGES - 1;
-      if (sn < nst) {
-        if (!mbar_wait(&empty[sn % FT_STAGES], ((sn / FT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        issue(sn, sn % FT_STAGES);
+    for (int st = 0; st < FT_STAGES - 1; ++st) {
+      if (st < nst && ok) {
+        const uint32_t f = done + st;
+        ok = mbar_wait(&empty[f % FT_STAGES], ((f / FT_STAGES) & 1) ^ 1, abort_flag);
+        if (ok) issue(st, f % FT_STAGES);
       }
       cp_async_commit();
-      cp_async_wait<FT_STAGES - 1>();                     // this thread's pieces of stage st have landed
-      const uint32_t sb = ring + (st % FT_STAGES) * FT_STAGE_BYTES;
+    }
+    for (int st = 0; ok && st < nst; ++st) {
+      const int sn = st + FT_STAGES - 1;
+      if (sn < nst) {
+        const uint32_t f = done + sn;
+        if (!mbar_wait(&empty[f % FT_STAGES], ((f / FT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        issue(sn, f % FT_STAGES);
+      }
+      cp_async_commit();
+      cp_async_wait<FT_STAGES - 1>();                     // this thread's pieces of fill st have landed
+      const uint32_t s_cur = (done + st) % FT_STAGES;
+      const uint32_t sb = ring + s_cur * FT_STAGE_BYTES;
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
         if (st * kps + kj[t] >= nk) continue;
@@ -406,7 +427,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       }
       fence_proxy_async();                                // cp.async writes -> visible to the tensor core
       __syncwarp();
-      if (lane == 0) mbar_arrive(&full[st % FT_STAGES]);
+      if (lane == 0) mbar_arrive(&full[s_cur]);
     }
     cp_async_wait<0>();
 
@@ -425,7 +446,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     named_barrier(1, FT_LOADERS);
 
     // ---- epilogue: thread = A row (TMEM lane); warps 0-3 scan columns 0-63, warps 4-7 columns 64-127
-    ok = ok && mbar_wait(acc_full, 0, abort_flag);
+    ok = ok && mbar_wait(acc_full, n_items & 1, abort_flag);
     ok = __all_sync(0xffffffffu, ok);                     // the TMEM loads below are warp-wide
     tc_fence_after();
     const int q = warp & 3, half = warp >> 2, row = q * 32 + lane, e = a0 + row;
@@ -467,14 +488,15 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         if (tl.blocks_b > 1) atomicMin(dst, key); else *dst = key;
       }
     }
+    tc_fence_before();                                    // TMEM reads done before the next tile's MMAs
   } else if (lane == 0) {
     // ---- MMA issue
     const uint32_t idesc = idesc_bf16(kFdTile, n_cols);
     const uint32_t chunk_step = passes == 4 ? 0u : (passes == 2 ? 16384u : 4096u);   // A block to A block
     const uint32_t b_from_a = passes == 2 ? 8192u : 16384u;
     for (int st = 0; st < nst; ++st) {
-      const int s = st % FT_STAGES;
-      if (!mbar_wait(&full[s], (st / FT_STAGES) & 1, abort_flag)) break;
+      const uint32_t f = done + st, s = f % FT_STAGES;
+      if (!mbar_wait(&full[s], (f / FT_STAGES) & 1, abort_flag)) break;
       tc_fence_after();
       for (int j = 0; j < kps && st * kps + j < nk; ++j) {
         const uint32_t sa = ring + s * FT_STAGE_BYTES + j * chunk_step;
@@ -487,6 +509,10 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     }
     umma_commit(acc_full);
   }
+  done += nst;
+  ++n_items;
+  if (*abort_flag) break;
+  }  // work items
   tc_fence_before();
   __syncthreads();
   if (warp == 8) {
@@ -498,16 +524,32 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
 
 bool tc_fd_supported(int hidden) { return hidden % 8 == 0; }
 
+// SMs of the current device (cached per device ordinal).
+static int sm_count() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (!cached[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 cudaError_t launch_fd_tc(const LayerLaunch& L) {
   const lightkv_layer_args_t* a = L.a;
   FdTcArgs f;
   f.x = static_cast<const __nv_bfloat16*>(a->hidden) + size_t(a->vis_begin) * a->hidden_row_stride;
-  f.batch_stride = a->hidden_batch_stride; f.row_stride = a->hidden_row_stride; f.d = L.hidden;
+  f.batch_stride = a->hidden_batch_stride; f.row_stride = a->hidden_row_stride; f.d = L.hidden; f.batch = L.batch;
   f.ws = L.ws; f.status = a->status;
   cudaError_t e = cudaFuncSetAttribute(fd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM);
   if (e != cudaSuccess) return e;
-  if (L.fd_tiles <= 0) return cudaSuccess;
-  fd_tc_kernel<<<dim3(L.fd_tiles, L.batch), FT_LOADERS + 32, FT_SMEM, L.stream>>>(f);
+  // persistent CTAs, two per SM, never more than there can be tiles
+  const long long bound = (long long)L.fd_tiles * L.batch;
+  if (bound <= 0) return cudaSuccess;
+  const int grid = (int)std::min<long long>(bound, 2LL * sm_count());
+  fd_tc_kernel<<<grid, FT_LOADERS + 32, FT_SMEM, L.stream>>>(f);
   return cudaGetLastError();
 }
 

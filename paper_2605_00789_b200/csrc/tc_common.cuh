@@ -40,17 +40,18 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait: gives up after ~2 s of wall time, raising *abort_flag (shared) so that every role
-// of the CTA unwinds; returns false on timeout or when another role already aborted.
+// of the CTA unwinds; returns false on timeout or when another role already aborted.  The clock is
+// only consulted every 4096 failed polls, so a wait that ends normally never reads it.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  uint32_t spins = 0;
-  while (true) {
+  uint64_t t0 = 0;
+  for (uint32_t spins = 1;; ++spins) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 0x3ff) == 0) {
+    if ((spins & 0xfff) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
     }
   }
 }
