@@ -250,26 +250,26 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
 // ======================================================================================================
 // FD + best partner on tensor cores (Eq. "similarity", Step 2).
 //
-// One CTA per tile of up to 128 A entries x 128 B entries (see FdTiling): a group of whole windows, or
-// one 128 x 128 block of a large window.  The rows of a tile are scattered over the sequence (they are
-// listed by a_tok / b_tok), so eight warps gather them with 16-byte cp.async copies, eight threads per
-// 128-byte row segment, straight into the 128-byte-swizzled K-major layout tcgen05 reads, through a
-// ring of three 32 KB stages.  A tile holds at most 32 * passes rows per operand (passes = 1, 2, 4), and
-// a stage holds 4 / passes consecutive 64-column chunks of both operands, so every thread always moves
-// eight 16-byte pieces per stage whatever the tile size, and two stages (64 KB) stay in flight per CTA,
-// two CTAs per SM.  Each thread re-reads the pieces it fetched to accumulate the rows' squared norms,
-// so X is read from HBM exactly once.  A ninth warp issues G += X_A X_B^T (128 x N x 64 per chunk,
-// N = B entries rounded up to 16, bf16 -> fp32 in TMEM).  The MMA always reads 128 A rows (16 KB) from
-// the start of a chunk's A block: rows the tile does not have are never written, overlap other blocks
-// of the same stage, and only feed accumulator rows nobody reads.  After the last chunk the loader
-// warps turn into the epilogue: one thread per A row scans the FD of the columns that belong to the
-// row's own window and keeps the minimum (ties: lowest B index).  Blocks of a large window combine
-// through a 64-bit atomicMin on (orderable FD, B index), which is order independent.
-//
-// Stage layout (offsets in KB), chosen so that the 16 KB A read stays inside the stage:
-//   passes 4: [A 0-16 | B 16-32]                     one chunk
-//   passes 2: [A0 0-8 | B0 8-16 | A1 16-24 | B1 24-32]   two chunks
-//   passes 1: [A0 A1 A2 A3 0-16 | B0 B1 B2 B3 16-32]     four chunks, 4 KB each
+// Persistent CTAs, two per SM; a work item is a tile of up to 128 A entries x 128 B entries (see
+// FdTiling): a group of whole windows, or one 128 x 128 block of a large window.  The rows of a tile are
+// scattered over the sequence (they are listed by a_tok / b_tok), so eight warps gather them with 16-byte
+// cp.async copies, eight threads per 128-byte row segment, straight into the 128-byte-swizzled K-major
+// layout tcgen05 reads.  The copies go through a ring of six 16 KB stages; a stage is 128 row slots of
+// 128 bytes (64 columns) and every loader thread fills four slots of it.  What the slots hold depends
+// on the tile's size (passes = 1, 2, 4 <=> at most 32, 64, 128 entries per operand):
+//   passes 4: even fills = the 128 A rows of a chunk, odd fills = its 128 B rows   (2 fills per chunk)
+//   passes 2: [64 A rows | 64 B rows] of one chunk                                  (1 fill per chunk)
+//   passes 1: [32 A rows, chunk c | 32 A rows, chunk c+1 | 32 B rows, c | 32 B rows, c+1]   (2 chunks per fill)
+// Four fills are in flight while a fifth is being consumed and a sixth may still be held by the tensor
+// core, so the loaders never wait for an MMA on their critical path.  Each thread re-reads the pieces
+// it fetched to accumulate the rows' squared norms: X is read from HBM exactly once.  A ninth warp
+// issues G += X_A X_B^T (128 x N x 64 per chunk, N = B entries rounded up to 16, bf16 -> fp32 in TMEM).
+// The MMA always reads 128 A rows (16 KB) from the start of a chunk's A block: rows the tile does not
+// have are never written, may overlap other blocks or the 4 KB pad behind the ring, and only feed
+// accumulator rows nobody reads.  After the last chunk the loader warps turn into the epilogue: one
+// thread per A row scans the FD of the columns that belong to the row's own window and keeps the
+// minimum (ties: lowest B index).  Blocks of a large window combine through a 64-bit atomicMin on
+// (orderable FD, B index), which is order independent.
 // ======================================================================================================
 struct FdTcArgs {
   const __nv_bfloat16* x;              // first vision row of sample 0
@@ -280,17 +280,19 @@ struct FdTcArgs {
 };
 
 constexpr int FT_LOADERS = 256;
-constexpr int FT_STAGES = 3;
-constexpr uint32_t FT_STAGE_BYTES = 32 * 1024;
-constexpr size_t FT_SMEM = size_t(FT_STAGES) * FT_STAGE_BYTES + 1024 /* alignment */ + 128 /* barriers */ +
+constexpr int FT_STAGES = 6;
+constexpr int FT_AHEAD = 4;                               // fills in flight
+constexpr uint32_t FT_STAGE_BYTES = 16 * 1024;
+constexpr uint32_t FT_RING_BYTES = FT_STAGES * FT_STAGE_BYTES + 4096;   // + pad for the 16 KB A read
+constexpr size_t FT_SMEM = size_t(FT_RING_BYTES) + 1024 /* alignment */ + 128 /* barriers */ +
                            4 * kFdTile * sizeof(float);
 
 __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(base + FT_STAGES * FT_STAGE_BYTES);
-  uint64_t* full = bars;                        // [FT_STAGES] stage landed (one arrival per loader warp)
-  uint64_t* empty = full + FT_STAGES;           // [FT_STAGES] stage consumed (MMA commit)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + FT_RING_BYTES);
+  uint64_t* full = bars;                        // [FT_STAGES] fill landed (one arrival per loader warp)
+  uint64_t* empty = full + FT_STAGES;           // [FT_STAGES] fill consumed (MMA commit)
   uint64_t* acc_full = empty + FT_STAGES;       // accumulator complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -315,9 +317,9 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   const int nW = a.ws.n_windows;
   const int nk = (a.d + 63) >> 6;               // 64-column chunks
 
-  // Persistent CTA: work items are the (sample, tile) pairs of the whole batch in sample order; this CTA
-  // takes items blockIdx.x, blockIdx.x + gridDim.x, ...  Barrier phases run on across items: `done` counts
-  // the stage fills this CTA has completed, `n_items` its finished tiles.
+  // Work items are the (sample, tile) pairs of the whole batch in sample order; this CTA takes items
+  // blockIdx.x, blockIdx.x + gridDim.x, ...  Barrier phases run on across items: `done` counts the
+  // fills this CTA has completed, `n_items` its finished tiles.
   uint32_t done = 0, n_items = 0;
   for (int item = blockIdx.x;; item += gridDim.x) {
   int b = 0, tile = item;
@@ -341,49 +343,51 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   const int b0 = win_off[w0] - a_off[w0] + ib * kFdTile, b1 = min(win_off[w1] - a_off[w1], b0 + cap_rows);
   if (a0 >= a1 || b0 >= b1) continue;           // same for every thread of the CTA
   const int n_cols = (b1 - b0 + 15) & ~15;      // MMA N
-  const int kps = 4 / passes;                   // chunks per stage
-  const int nst = (nk + kps - 1) / kps;         // stage fills of this tile
+  const int nf = passes == 4 ? 2 * nk : (passes == 2 ? nk : (nk + 1) >> 1);   // fills of this tile
 
   if (warp < 8) {
-    // ---- gather: thread = 16-byte piece c of rows g + 32 i (i < passes) of both operands, for every chunk
-    //      of the stage; copy t of a stage is (chunk t / passes, row g + 32 (t % passes))
+    // ---- gather: thread = 16-byte piece c of row slots g, g + 32, g + 64, g + 96 of every fill
     const int c = tid & 7, g = tid >> 3;
     const unsigned char* xb = reinterpret_cast<const unsigned char*>(a.x + size_t(b) * a.batch_stride);
     const int* a_tok = a.ws.a_tok + size_t(b) * a.ws.cap_a;
     const int* b_tok = a.ws.b_tok + size_t(b) * a.ws.cap_b;
-    const uint32_t piece = uint32_t(g) * 128 + (uint32_t(c ^ (g & 7)) << 4);   // swizzled offset inside a block
-    const unsigned char* ap[4];
-    const unsigned char* bp[4];
-    uint32_t a_so[4], b_so[4];                            // shared-memory offset of copy t inside a stage
-    int kj[4];                                            // chunk of copy t inside a stage
-    uint32_t a_ok = 0, b_ok = 0;
+    // source row of slot t on even / odd fills (they differ only when passes = 4), validity bits, and the
+    // chunk of slot t relative to the fill's first chunk (passes = 1 packs two chunks into a fill)
+    const unsigned char* src_e[4];
+    const unsigned char* src_o[4];
+    uint32_t ok_e = 0, ok_o = 0;
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
-      const int i = t & (passes - 1), j = t / passes;
+      const int i = passes == 4 ? t : (passes == 2 ? (t & 1) : 0);          // row g + 32 i of the operand
+      const bool slot_b = passes == 4 ? false : (t >> 1) != 0;              // operand of slot t on even fills
       const int ea = a0 + g + 32 * i, eb = b0 + g + 32 * i;
       const int ta = ea < a1 ? a_tok[ea] : -1, tb = eb < b1 ? b_tok[eb] : -1;
-      a_ok |= (ta >= 0 ? 1u : 0u) << t;
-      b_ok |= (tb >= 0 ? 1u : 0u) << t;
-      ap[t] = xb + (size_t(max(ta, 0)) * a.row_stride + c * 8) * 2 + size_t(j) * 128;
-      bp[t] = xb + (size_t(max(tb, 0)) * a.row_stride + c * 8) * 2 + size_t(j) * 128;
-      kj[t] = j;
-      if (passes == 2) { a_so[t] = j * 16384 + i * 4096 + piece; b_so[t] = a_so[t] + 8192; }
-      else { a_so[t] = t * 4096 + piece; b_so[t] = 16384 + t * 4096 + piece; }
+      const unsigned char* pa = xb + (size_t(max(ta, 0)) * a.row_stride + c * 8) * 2;
+      const unsigned char* pb = xb + (size_t(max(tb, 0)) * a.row_stride + c * 8) * 2;
+      const size_t sub = passes == 1 ? size_t(t & 1) * 128 : 0;             // second chunk of the fill
+      src_e[t] = (slot_b ? pb : pa) + sub;
+      src_o[t] = (passes == 4 ? pb : (slot_b ? pb : pa)) + sub;
+      ok_e |= ((slot_b ? tb : ta) >= 0 ? 1u : 0u) << t;
+      ok_o |= ((passes == 4 ? tb : (slot_b ? tb : ta)) >= 0 ? 1u : 0u) << t;
     }
-    float ssa[4] = {0.f, 0.f, 0.f, 0.f}, ssb[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t slot0 = uint32_t(g) * 128 + (uint32_t(c ^ (g & 7)) << 4);   // swizzled offset of slot g; slot g+32t is 4096 t further
+    const int chunk_shift = passes == 4 ? 1 : 0, chunk_mul = passes == 1 ? 2 : 1;
+    float acc_e[4] = {0.f, 0.f, 0.f, 0.f}, acc_o[4] = {0.f, 0.f, 0.f, 0.f};
 
     // rows the tile does not have and chunks past the hidden size are not fetched at all; the pieces of
     // the last chunk that lie past the hidden size are zero-filled
-    auto issue = [&](int st, int stage) {
-      const uint32_t sb = ring + stage * FT_STAGE_BYTES;
-      const size_t koff = size_t(st) * kps * 128;
+    auto issue = [&](int f, uint32_t stage) {
+      const uint32_t sb = ring + stage * FT_STAGE_BYTES + slot0;
+      const bool odd = passes == 4 && (f & 1);
+      const int kc0 = (f >> chunk_shift) * chunk_mul;
+      const uint32_t okm = odd ? ok_o : ok_e;
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
-        const int kc = st * kps + kj[t];
-        if (kc >= nk) continue;
+        const int kc = kc0 + (passes == 1 ? (t & 1) : 0);
+        if (kc >= nk || !((okm >> t) & 1)) continue;
         const uint32_t bytes = (kc * 64 + c * 8 < a.d) ? 16u : 0u;   // d is a multiple of 8
-        if ((a_ok >> t) & 1) cp_async16(sb + a_so[t], ap[t] + (bytes ? koff : 0), bytes);
-        if ((b_ok >> t) & 1) cp_async16(sb + b_so[t], bp[t] + (bytes ? koff : 0), bytes);
+        const unsigned char* p = odd ? src_o[t] : src_e[t];
+        cp_async16(sb + t * 4096, p + (bytes ? size_t(kc0) * 128 : 0), bytes);
       }
     };
     auto sumsq = [](const uint4& v, float acc) {
@@ -397,33 +401,36 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       return acc;
     };
 
-    // fill f of this CTA (counted across tiles) uses stage f % 3; it may be written once the MMAs of fill
-    // f - 3 have completed, and is complete for the MMA warp on phase (f / 3) & 1 of full[]
+    // fill F of this CTA (counted across tiles) uses stage F % 6; it may be written once the MMAs that read
+    // fill F - 6 have completed, and is complete for the MMA warp on phase (F / 6) & 1 of full[]
     bool ok = true;
-    for (int st = 0; st < FT_STAGES - 1; ++st) {
-      if (st < nst && ok) {
-        const uint32_t f = done + st;
-        ok = mbar_wait(&empty[f % FT_STAGES], ((f / FT_STAGES) & 1) ^ 1, abort_flag);
-        if (ok) issue(st, f % FT_STAGES);
+    for (int f = 0; f < FT_AHEAD; ++f) {
+      if (f < nf && ok) {
+        const uint32_t F = done + f;
+        ok = mbar_wait(&empty[F % FT_STAGES], ((F / FT_STAGES) & 1) ^ 1, abort_flag);
+        if (ok) issue(f, F % FT_STAGES);
       }
       cp_async_commit();
     }
-    for (int st = 0; ok && st < nst; ++st) {
-      const int sn = st + FT_STAGES - 1;
-      if (sn < nst) {
-        const uint32_t f = done + sn;
-        if (!mbar_wait(&empty[f % FT_STAGES], ((f / FT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        issue(sn, f % FT_STAGES);
+    for (int f = 0; ok && f < nf; ++f) {
+      const int fn = f + FT_AHEAD;
+      if (fn < nf) {
+        const uint32_t F = done + fn;
+        if (!mbar_wait(&empty[F % FT_STAGES], ((F / FT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        issue(fn, F % FT_STAGES);
       }
       cp_async_commit();
-      cp_async_wait<FT_STAGES - 1>();                     // this thread's pieces of fill st have landed
-      const uint32_t s_cur = (done + st) % FT_STAGES;
-      const uint32_t sb = ring + s_cur * FT_STAGE_BYTES;
+      cp_async_wait<FT_AHEAD>();                          // this thread's pieces of fill f have landed
+      const uint32_t s_cur = (done + f) % FT_STAGES;
+      const uint32_t sb = ring + s_cur * FT_STAGE_BYTES + slot0;
+      const bool odd = passes == 4 && (f & 1);
+      const int kc0 = (f >> chunk_shift) * chunk_mul;
+      const uint32_t okm = odd ? ok_o : ok_e;
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
-        if (st * kps + kj[t] >= nk) continue;
-        if ((a_ok >> t) & 1) ssa[t] = sumsq(ld_shared16(sb + a_so[t]), ssa[t]);
-        if ((b_ok >> t) & 1) ssb[t] = sumsq(ld_shared16(sb + b_so[t]), ssb[t]);
+        if (kc0 + (passes == 1 ? (t & 1) : 0) >= nk || !((okm >> t) & 1)) continue;
+        const uint4 v = ld_shared16(sb + t * 4096);
+        if (odd) acc_o[t] = sumsq(v, acc_o[t]); else acc_e[t] = sumsq(v, acc_e[t]);
       }
       fence_proxy_async();                                // cp.async writes -> visible to the tensor core
       __syncwarp();
@@ -431,9 +438,12 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     }
     cp_async_wait<0>();
 
-    // ---- norms: copies of the same row, then the eight threads of a row, hold partial sums
-    if (passes == 2) { ssa[0] += ssa[2]; ssa[1] += ssa[3]; ssb[0] += ssb[2]; ssb[1] += ssb[3]; }
-    if (passes == 1) { ssa[0] += ssa[1] + ssa[2] + ssa[3]; ssb[0] += ssb[1] + ssb[2] + ssb[3]; }
+    // ---- norms: squared sums of A row g + 32 i and B row g + 32 i, then across the eight threads of a row
+    float ssa[4], ssb[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { ssa[i] = acc_e[i]; ssb[i] = acc_o[i]; }                 // passes 4
+    if (passes == 2) { ssb[0] = acc_e[2]; ssb[1] = acc_e[3]; }
+    if (passes == 1) { ssa[0] = acc_e[0] + acc_e[1]; ssb[0] = acc_e[2] + acc_e[3]; }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
 #pragma unroll
@@ -490,26 +500,42 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     }
     tc_fence_before();                                    // TMEM reads done before the next tile's MMAs
   } else if (lane == 0) {
-    // ---- MMA issue
+    // ---- MMA issue: one chunk = four K = 16 steps inside the 128-byte rows
     const uint32_t idesc = idesc_bf16(kFdTile, n_cols);
-    const uint32_t chunk_step = passes == 4 ? 0u : (passes == 2 ? 16384u : 4096u);   // A block to A block
-    const uint32_t b_from_a = passes == 2 ? 8192u : 16384u;
-    for (int st = 0; st < nst; ++st) {
-      const uint32_t f = done + st, s = f % FT_STAGES;
-      if (!mbar_wait(&full[s], (f / FT_STAGES) & 1, abort_flag)) break;
-      tc_fence_after();
-      for (int j = 0; j < kps && st * kps + j < nk; ++j) {
-        const uint32_t sa = ring + s * FT_STAGE_BYTES + j * chunk_step;
+    auto chunk_mma = [&](uint32_t a_addr, uint32_t b_addr, bool first) {
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          umma_bf16(tmem_base, smem_desc_sw128(sa + kk * 32), smem_desc_sw128(sa + b_from_a + kk * 32), idesc,
-                    (st | j | kk) != 0);
+      for (int kk = 0; kk < 4; ++kk)
+        umma_bf16(tmem_base, smem_desc_sw128(a_addr + kk * 32), smem_desc_sw128(b_addr + kk * 32), idesc,
+                  !(first && kk == 0));
+    };
+    if (passes == 4) {
+      for (int k = 0; k < nk; ++k) {
+        const uint32_t FA = done + 2 * k, FB = FA + 1, sA = FA % FT_STAGES, sB = FB % FT_STAGES;
+        if (!mbar_wait(&full[sA], (FA / FT_STAGES) & 1, abort_flag)) break;
+        if (!mbar_wait(&full[sB], (FB / FT_STAGES) & 1, abort_flag)) break;
+        tc_fence_after();
+        chunk_mma(ring + sA * FT_STAGE_BYTES, ring + sB * FT_STAGE_BYTES, k == 0);
+        umma_commit(&empty[sA]);
+        umma_commit(&empty[sB]);
       }
-      umma_commit(&empty[s]);
+    } else {
+      for (int f = 0; f < nf; ++f) {
+        const uint32_t F = done + f, s = F % FT_STAGES;
+        if (!mbar_wait(&full[s], (F / FT_STAGES) & 1, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t sa = ring + s * FT_STAGE_BYTES;
+        if (passes == 2) {
+          chunk_mma(sa, sa + 8192, f == 0);
+        } else {
+          chunk_mma(sa, sa + 8192, f == 0);
+          if (2 * f + 1 < nk) chunk_mma(sa + 4096, sa + 12288, false);
+        }
+        umma_commit(&empty[s]);
+      }
     }
     umma_commit(acc_full);
   }
-  done += nst;
+  done += nf;
   ++n_items;
   if (*abort_flag) break;
   }  // work items
