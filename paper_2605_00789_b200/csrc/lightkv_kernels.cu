@@ -474,6 +474,7 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
 // =====================================================================================================
 struct SelectArgs {
   int n_q_heads, xi_mode, cap_out;
+  int smem_tokens;                    // tokens the dynamic shared memory has room for (0: use the workspace)
   double keep;
   const int* n_vis;
   const int* pos;
@@ -528,9 +529,13 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   const int* a_win = ws.a_win + size_t(b) * ws.cap_a;
   const unsigned long long* a_key = ws.a_key + size_t(b) * ws.cap_a;
   const int* b_tok = ws.b_tok + size_t(b) * ws.cap_b;
-  float* xi = ws.xi + size_t(b) * ws.cap_in;
-  int* partner = ws.partner + size_t(b) * ws.cap_in;
-  int* slot = ws.slot + size_t(b) * ws.cap_in;
+  // xi, partner and slot are read back through dependent chains in phases 2-5: keep them in shared
+  // memory when the sample fits (the launch passes 12 bytes per token), else in the workspace
+  extern __shared__ __align__(16) unsigned char select_smem[];
+  const bool in_smem = a.smem_tokens >= ws.cap_in;
+  float* xi = in_smem ? reinterpret_cast<float*>(select_smem) : ws.xi + size_t(b) * ws.cap_in;
+  int* partner = in_smem ? reinterpret_cast<int*>(select_smem) + ws.cap_in : ws.partner + size_t(b) * ws.cap_in;
+  int* slot = in_smem ? reinterpret_cast<int*>(select_smem) + 2 * ws.cap_in : ws.slot + size_t(b) * ws.cap_in;
   const int* pos = a.pos ? a.pos + size_t(b) * ws.cap_in : nullptr;
   int* dst = a.dst + size_t(b) * ws.cap_in;
   float* weight = a.weight + size_t(b) * ws.cap_in;
@@ -545,6 +550,7 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     else if (a.xi_mode == LIGHTKV_XI_UNIFORM) v = 1.0f;
     else {
       v = 0.f;
+#pragma unroll 8
       for (int h = 0; h < a.n_q_heads; ++h) v += ws.xi_h[(size_t(b) * a.n_q_heads + h) * ws.cap_in + i];
     }
     xi[i] = v;
@@ -654,7 +660,13 @@ cudaError_t launch_select_map(const LayerLaunch& L) {
   s.n_vis = a->n_vis; s.pos = a->pos; s.xi_in = a->xi; s.n_vis_out = a->n_vis_out; s.pos_out = a->pos_out;
   s.dst = a->dst; s.weight = a->weight; s.grp_off = a->grp_off; s.grp_src = a->grp_src;
   s.xi_out = a->xi_out; s.status = a->status;
-  select_map_kernel<<<L.batch, 1024, 0, L.stream>>>(L.ws, s);
+  constexpr int kSelectSmemTokens = 16384;               // 12 bytes per token -> 192 KB
+  const size_t smem = L.ws.cap_in <= kSelectSmemTokens ? size_t(L.ws.cap_in) * 12 : 0;
+  s.smem_tokens = smem ? L.ws.cap_in : 0;
+  cudaError_t e = cudaFuncSetAttribute(select_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSelectSmemTokens * 12);
+  if (e != cudaSuccess) return e;
+  select_map_kernel<<<L.batch, 1024, smem, L.stream>>>(L.ws, s);
   return cudaGetLastError();
 }
 
@@ -743,7 +755,7 @@ cudaError_t launch_merge_rows(const LayerLaunch& L) {
 // K/V merge-compaction ("key and value tokens are compressed simultaneously for later layers").
 // The stage's merge map is applied per KV head; contiguous (strided) or paged (block-table) addressing
 // on either side.  A CTA takes a few consecutive output tokens (as many as give its threads four
-// 16-byte units each).  It first resolves, once per token, where the token goes and which source
+// rounds of four 16-byte units each).  It first resolves, once per token, where the token goes and which source
 // tokens feed it with which weight (shared memory), then every thread issues the loads of all its
 // units back to back before it touches any of them, so that each thread keeps up to eight 16-byte
 // loads in flight.  Groups of one are copied; larger groups are summed in fp32 in member order.
@@ -759,7 +771,7 @@ struct KvAddr {
   }
 };
 
-constexpr int KV_THREADS = 256, KV_ITEMS = 4, KV_MAXM = 8, KV_MAXROWS = 8;
+constexpr int KV_THREADS = 256, KV_ITEMS = 4, KV_MAXM = 8, KV_MAXROWS = 32, KV_BATCHES = 4;
 
 template <typename T>
 __global__ void __launch_bounds__(KV_THREADS)
@@ -868,7 +880,8 @@ cudaError_t launch_kv_compact(const KvLaunch& K) {
   KvAddr da{a->dst_batch_stride, a->dst_head_stride, a->dst_row_stride, a->dst_page_stride,
             a->page_size > 0 ? a->dst_block_table : nullptr, a->page_size, a->max_blocks};
   const int units = 2 * K.n_kv_heads * (K.head_dim * (K.dtype == LIGHTKV_BF16 ? 2 : 4) / 16);
-  const int rows_per_cta = std::max(1, std::min(KV_MAXROWS, KV_THREADS * KV_ITEMS / units));
+  // a CTA resolves the metadata of its tokens once and then moves about KV_BATCHES x 1024 units
+  const int rows_per_cta = std::max(1, std::min(KV_MAXROWS, KV_BATCHES * KV_THREADS * KV_ITEMS / units));
   const int rows = a->vis_begin + K.cap_out + a->n_text_after;
   const dim3 grid((rows + rows_per_cta - 1) / rows_per_cta, K.batch);
   const int gather = a->mode == LIGHTKV_KV_GATHER;
