@@ -34,8 +34,12 @@ import lightkv_synth as S  # noqa: E402
 KERNELS = ("window_build", "xi", "fd_best_partner", "select_map", "merge_hidden", "kv_compact")
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
-# keyed by (workload, kernel); null until a capture exists for that pair.
-NCU_TRAFFIC_BYTES = {}
+# of the stage-0 launch, keyed by (workload, kernel); null where no capture exists.
+NCU_TRAFFIC_BYTES = {
+    ("cfg2", "xi"): 391.76e6,                # profiles/xi_tc_kernel_cfg2_stage0.txt
+    ("cfg2", "fd_best_partner"): 193.17e6,   # profiles/fd_tc_kernel_cfg2_stage0.txt
+    ("cfg2", "merge_hidden"): 264.45e6,      # profiles/merge_rows_kernel_cfg2_stage0.txt
+}
 
 
 def measured_peaks():
@@ -123,7 +127,7 @@ def whole_job_throughput(tokens_per_rank_step: int, world: int, ms_step_max: flo
 
 # ------------------------------------------------------------------------------------------ workload
 
-def build_inputs(wl, plan, L, torch, device, sample_offset):
+def build_inputs(wl, plan, L, torch, device, sample_offset, kv_layout="bhnd"):
     """Generate every stage's inputs on the host (pinned) and upload them.  Stage i+1 is sampled at the
     positions that survive stage i (taken from one untimed run of the library itself)."""
     samples = rank_samples(sample_offset // wl.batch, wl.batch)
@@ -135,7 +139,12 @@ def build_inputs(wl, plan, L, torch, device, sample_offset):
         for name in ("hidden", "q", "k", "v"):
             t = torch.from_numpy(S.bf16_bits(inp[name]).view(np.int16)).view(torch.bfloat16).pin_memory()
             host[name] = t
-            dev[name] = t.to(device, non_blocking=True)
+            if name in ("k", "v") and kv_layout == "bnhd":      # token-major cache, handed over as a strided view
+                store = torch.empty((t.shape[0], t.shape[2], t.shape[1], t.shape[3]), dtype=t.dtype, device=device)
+                dev[name] = store.permute(0, 2, 1, 3)
+                dev[name].copy_(t, non_blocking=True)
+            else:
+                dev[name] = t.to(device, non_blocking=True)
         n_seq = host["hidden"].shape[1]
         pos_pad = np.full((wl.batch, info.cap_in), -1, dtype=np.int32)
         pos_pad[:, :inp["pos"].shape[1]] = inp["pos"]
@@ -143,8 +152,14 @@ def build_inputs(wl, plan, L, torch, device, sample_offset):
         dev["n_vis"] = torch.from_numpy(inp["n_vis"]).to(device)
         n_seq_out = wl.n_text + info.cap_out
         out = L.StageBuffers(plan, st, n_seq_out, device)
-        k_dst = torch.empty((wl.batch, wl.n_kv_heads, n_seq_out, wl.head_dim), dtype=torch.bfloat16, device=device)
-        v_dst = torch.empty_like(k_dst)
+        if kv_layout == "bnhd":
+            k_dst = torch.empty((wl.batch, n_seq_out, wl.n_kv_heads, wl.head_dim), dtype=torch.bfloat16,
+                                device=device).permute(0, 2, 1, 3)
+            v_dst = torch.empty((wl.batch, n_seq_out, wl.n_kv_heads, wl.head_dim), dtype=torch.bfloat16,
+                                device=device).permute(0, 2, 1, 3)
+        else:
+            k_dst = torch.empty((wl.batch, wl.n_kv_heads, n_seq_out, wl.head_dim), dtype=torch.bfloat16, device=device)
+            v_dst = torch.empty_like(k_dst)
         host_out = {"hidden": torch.empty(out.hidden_out.shape, dtype=torch.bfloat16).pin_memory(),
                     "k": torch.empty(k_dst.shape, dtype=torch.bfloat16).pin_memory(),
                     "v": torch.empty(k_dst.shape, dtype=torch.bfloat16).pin_memory(),
@@ -164,43 +179,58 @@ def build_inputs(wl, plan, L, torch, device, sample_offset):
     return stages
 
 
-def run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None):
+def run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None, side=None):
+    """lightkv_compress_layer on the current stream, then lightkv_compact_kv either on the same stream or,
+    when `side` is given, on that stream behind an event (the compaction only needs the stage's merge map)."""
+    import torch
     d = stg["dev"]
     L.compress_layer(plan, st, d["hidden"], stg["out"], vis_begin=wl.n_text, q=d["q"], k=d["k"], n_vis=n_vis,
                      pos=pos, trace_events=trace)
-    L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
-                 n_vis=n_vis)
+    if side is None:
+        L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
+                     n_vis=n_vis)
+    else:
+        side.wait_stream(torch.cuda.current_stream())
+        L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
+                     n_vis=n_vis, stream=side)
 
 
-def run_step(L, plan, wl, stages, traces=None, kv_events=None):
-    """The whole hot path once; stage i+1 reads positions and counts stage i left on the device."""
+def run_step(L, plan, wl, stages, traces=None, kv_events=None, side=None):
+    """The whole hot path once; stage i+1 reads positions and counts stage i left on the device.
+    With `side`, the K/V compaction of stage i (HBM bound) runs on that second stream while stage i+1's
+    compression (bound by the xi contraction) proceeds on the current one; the step ends with a join."""
+    import torch
     pos, n_vis = stages[0]["dev"]["pos"], stages[0]["dev"]["n_vis"]
     for st, stg in enumerate(stages):
-        run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None if traces is None else traces[st])
+        run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None if traces is None else traces[st], side=side)
         if kv_events is not None:
             kv_events[st].record()
         pos, n_vis = stg["out"].pos_out, stg["out"].n_vis_out
+    if side is not None:
+        torch.cuda.current_stream().wait_stream(side)
 
 
 def algorithmic_work(wl, stages):
-    """Per kernel, summed over the stages of one step: algorithmic bytes (HBM streams) or flops (xi)."""
+    """Per stage and per kernel: algorithmic bytes (HBM streams) or flops (xi) of one launch."""
     e = 2  # bf16
-    work = {k: 0.0 for k in KERNELS}
+    per_stage = []
     nt = wl.n_text
     for stg in stages:
+        work = {}
         n_in = stg["n_vis"].astype(np.float64)
         n_out = stg["n_out"].astype(np.float64)
         # xi, ATTN_FULL: 2*dh flops per (head, query, visible key); query t sees n_text + t + 1 keys
-        work["xi"] += float((2.0 * wl.n_q_heads * wl.head_dim * (n_in * (nt + 1) + n_in * (n_in - 1) / 2)).sum())
+        work["xi"] = float((2.0 * wl.n_q_heads * wl.head_dim * (n_in * (nt + 1) + n_in * (n_in - 1) / 2)).sum())
         # FD: one read of the vision rows (+ 8 bytes of keys per A node)
-        work["fd_best_partner"] += float((n_in * wl.hidden * e + 4 * n_in).sum())
+        work["fd_best_partner"] = float((n_in * wl.hidden * e + 4 * n_in).sum())
         # hidden merge: every input row read once, every output row written once
-        work["merge_hidden"] += float(((nt + n_in) * wl.hidden * e + (nt + n_out) * wl.hidden * e).sum())
+        work["merge_hidden"] = float(((nt + n_in) * wl.hidden * e + (nt + n_out) * wl.hidden * e).sum())
         # K/V: same for K and V, all KV heads
-        work["kv_compact"] += float((2 * wl.n_kv_heads * wl.head_dim * e * ((nt + n_in) + (nt + n_out))).sum())
-        work["window_build"] += float((n_in * 4 * 5).sum())
-        work["select_map"] += float((n_in * 4 * 10).sum())
-    return work
+        work["kv_compact"] = float((2 * wl.n_kv_heads * wl.head_dim * e * ((nt + n_in) + (nt + n_out))).sum())
+        work["window_build"] = float((n_in * 4 * 5).sum())
+        work["select_map"] = float((n_in * 4 * 10).sum())
+        per_stage.append(work)
+    return per_stage
 
 
 def oracle_sample_step(wl, full_schedule=True):
@@ -250,6 +280,10 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(S.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--engine", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--kv-layout", default="bhnd", choices=["bhnd", "bnhd"],
+                    help="K/V cache layout: [B,H_kv,N,dh] (head-major) or [B,N,H_kv,dh] (token-major)")
+    ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
+                    help="2: K/V compaction of stage i on a second stream, overlapping stage i+1's compression")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -263,7 +297,7 @@ def main():
     config = {"workload": f"{wl.name}: {wl.n_stages}-stage schedule layers={list(wl.layers)} windows={list(wl.windows)} "
                           f"keep={list(wl.keep)}, batch {wl.batch}, {wl.n_vis} vision + {wl.n_text} text tokens, "
                           f"hidden {wl.hidden}, {wl.n_q_heads}q/{wl.n_kv_heads}kv heads x {wl.head_dim}, "
-                          f"xi from full causal attention, K/V merge",
+                          f"xi from full causal attention, K/V merge, K/V layout {args.kv_layout}",
               "l2": "inputs larger than L2 (every stage streams > 126 MB)", "batch_per_gpu": wl.batch}
 
     if args.impl == "reference":
@@ -307,7 +341,7 @@ def main():
     plan = L.Plan(wl.batch, wl.hidden, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_layers, wl.tiles, wl.layers,
                   wl.windows, wl.keep, wl.n_text, dtype=L.BF16, xi_mode=L.XI_ATTN_FULL,
                   engine=L.ENGINE_AUTO if args.engine == "auto" else L.ENGINE_SIMT)
-    stages = build_inputs(wl, plan, L, torch, device, sample_offset=rank * wl.batch)
+    stages = build_inputs(wl, plan, L, torch, device, sample_offset=rank * wl.batch, kv_layout=args.kv_layout)
     tokens_per_step = int(sum(int(s["n_vis"].sum()) for s in stages))
     n_stages = len(stages)
 
@@ -316,22 +350,23 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    side = torch.cuda.Stream(device=device) if args.streams == 2 else None
     for _ in range(args.warmup):
-        run_step(L, plan, wl, stages)
-    # per-kernel events inside the timed region: TRACE_EVENTS per (step, stage) + one after compact_kv
+        run_step(L, plan, wl, stages, side=side)
+
     def ev():
         e = torch.cuda.Event(enable_timing=True)
         e.record()                    # torch creates the CUDA event lazily; the C ABI needs a live handle
         return e
-    traces = [[[ev() for _ in range(L.TRACE_EVENTS)] for _ in range(n_stages)] for _ in range(args.steps)]
-    kv_ev = [[ev() for _ in range(n_stages)] for _ in range(args.steps)]
+    # timed region: K whole steps in the benchmark's schedule (--streams 2: K/V compaction of a stage on a
+    # second stream, overlapping the next stage's compression)
     t_begin, t_end = ev(), ev()
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
     t_begin.record()
     for i in range(args.steps):
-        run_step(L, plan, wl, stages, traces[i], kv_ev[i])
+        run_step(L, plan, wl, stages, side=side)
     t_end.record()
     barrier()
     clocks = sampler.stop()
@@ -339,33 +374,61 @@ def main():
     ms_step = ms_total / args.steps
     value = whole_job_throughput(tokens_per_step, world, ms_step)
 
+    # per-kernel pass: the same steps on ONE stream, with the library's trace events between its launches
+    # (TRACE_EVENTS per (step, stage) + one after compact_kv), so that every kernel is timed alone
+    ksteps = max(3, min(args.steps, 10))
+    traces = [[[ev() for _ in range(L.TRACE_EVENTS)] for _ in range(n_stages)] for _ in range(ksteps)]
+    kv_ev = [[ev() for _ in range(n_stages)] for _ in range(ksteps)]
+    k_begin, k_end = ev(), ev()
+    barrier()
+    k_begin.record()
+    for i in range(ksteps):
+        run_step(L, plan, wl, stages, traces[i], kv_ev[i])
+    k_end.record()
+    barrier()
+    ms_step_one_stream = max_over_ranks(k_begin.elapsed_time(k_end), world, device) / ksteps
+
     ktime = {k: 0.0 for k in KERNELS}       # ms per step, summed over stages
     kstage = [{k: 0.0 for k in KERNELS} for _ in range(n_stages)]
-    for i in range(args.steps):
+    for i in range(ksteps):
         for st in range(n_stages):
             e = traces[i][st]
             for j, name in enumerate(L.TRACE_NAMES):
-                kstage[st][name] += e[j].elapsed_time(e[j + 1]) / args.steps
-            kstage[st]["kv_compact"] += e[-1].elapsed_time(kv_ev[i][st]) / args.steps
+                kstage[st][name] += e[j].elapsed_time(e[j + 1]) / ksteps
+            kstage[st]["kv_compact"] += e[-1].elapsed_time(kv_ev[i][st]) / ksteps
     for st in range(n_stages):
         for k in KERNELS:
             ktime[k] += kstage[st][k]
-    work = algorithmic_work(wl, stages)
+    work_stage = algorithmic_work(wl, stages)
+    work = {k: sum(w[k] for w in work_stage) for k in KERNELS}
     peaks = measured_peaks()
+
+    def rate(k, amount, ms):
+        sec = ms / 1e3
+        if k == "xi":
+            return amount / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", "tensor"
+        return amount / sec / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+
     kernels = {}
     for k in KERNELS:
-        sec = ktime[k] / 1e3
-        if k == "xi":
-            ach, peak, u, bound = work[k] / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", "tensor"
-        else:
-            ach, peak, u, bound = work[k] / sec / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+        ach, peak, u, bound = rate(k, work[k], ktime[k])
         kernels[k] = {"ms_per_step": round(ktime[k], 4), "share": round(ktime[k] / sum(ktime.values()), 4),
                       "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": u, "frac": round(ach / peak, 4)}
+    # roofline object: the kernel with the largest share, at its largest launch (stage 0), so that `achieved`
+    # and `traffic` are both per launch
     top = max(KERNELS, key=lambda k: ktime[k])
-    roofline = {"kernel": top, "bound": kernels[top]["bound"], "achieved": kernels[top]["achieved"],
-                "peak": kernels[top]["peak"], "unit": kernels[top]["unit"], "frac": kernels[top]["frac"],
-                "traffic": NCU_TRAFFIC_BYTES.get((wl.name, top)), "peak_source": f"of {peaks['source']}",
-                "launches_per_step": n_stages}
+    ach, peak, u, bound = rate(top, work_stage[0][top], kstage[0][top])
+    roofline = {"kernel": top, "launch": "stage 0", "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": u,
+                "frac": round(ach / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get((wl.name, top)),
+                "algorithmic": work_stage[0][top], "us": round(1e3 * kstage[0][top], 1),
+                "peak_source": f"of {peaks['source']}"}
+    if top == "xi":
+        # one exponential per logit on the special-function unit (16 per clock per SM) is the narrower bound
+        logits = work_stage[0]["xi"] / (2.0 * wl.head_dim)
+        sfu_peak = 16.0 * 148 * 1.965e9
+        roofline["sfu"] = {"achieved_exp_per_s": logits / (kstage[0]["xi"] / 1e3), "peak_exp_per_s": sfu_peak,
+                           "frac": round(logits / (kstage[0]["xi"] / 1e3) / sfu_peak, 4),
+                           "note": "16 ex2/clk/SM x 148 SMs x 1.965 GHz"}
 
     # end to end through the public API with host buffers: H2D of every stage's inputs from pinned
     # memory, the step, D2H of every stage's results
@@ -378,7 +441,7 @@ def main():
             for st, s in enumerate(stages):
                 for name, t in s["host"].items():
                     s["dev"][name].copy_(t, non_blocking=True)
-            run_step(L, plan, wl, stages)
+            run_step(L, plan, wl, stages, side=side)
             for s in stages:
                 s["host_out"]["hidden"].copy_(s["out"].hidden_out, non_blocking=True)
                 s["host_out"]["k"].copy_(s["k_dst"], non_blocking=True)
@@ -411,6 +474,9 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
                 "us_per_compression_layer": 1e3 * ms_step / n_stages,
+                "schedule": ("two streams: lightkv_compact_kv of stage i overlaps lightkv_compress_layer of stage i+1"
+                             if side is not None else "one stream"),
+                "ms_per_step_one_stream": ms_step_one_stream,
                 "roofline": roofline, "kernels": kernels,
                 "us_by_stage": [{k: round(1e3 * v, 1) for k, v in ks.items()} for ks in kstage], "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                 "gpu_launches": launches_per_step * args.steps,

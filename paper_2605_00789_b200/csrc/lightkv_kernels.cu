@@ -754,11 +754,10 @@ cudaError_t launch_merge_rows(const LayerLaunch& L) {
 // =====================================================================================================
 // K/V merge-compaction ("key and value tokens are compressed simultaneously for later layers").
 // The stage's merge map is applied per KV head; contiguous (strided) or paged (block-table) addressing
-// on either side.  A CTA takes a few consecutive output tokens (as many as give its threads four
-// rounds of four 16-byte units each).  It first resolves, once per token, where the token goes and which source
-// tokens feed it with which weight (shared memory), then every thread issues the loads of all its
-// units back to back before it touches any of them, so that each thread keeps up to eight 16-byte
-// loads in flight.  Groups of one are copied; larger groups are summed in fp32 in member order.
+// on either side.  One CTA per output token, small enough in registers for six CTAs per SM; every thread
+// resolves the token's group itself (uniform, cached loads) and keeps the loads of up to four group
+// members in flight per 16-byte unit.  Groups of one are copied; larger groups are summed in fp32 in
+// member order.
 // =====================================================================================================
 struct KvAddr {
   int64_t batch_stride, head_stride, row_stride, page_stride;
@@ -771,105 +770,73 @@ struct KvAddr {
   }
 };
 
-constexpr int KV_THREADS = 256, KV_ITEMS = 4, KV_MAXM = 8, KV_MAXROWS = 32, KV_BATCHES = 4;
+constexpr int KV_THREADS = 256;
+
+// floor(n / d) for n, d < 65536 with m = ceil(2^32 / d): one multiply instead of a division
+__device__ inline int div_magic(int n, unsigned m) { return (int)__umulhi((unsigned)n, m); }
 
 template <typename T>
-__global__ void __launch_bounds__(KV_THREADS)
+__global__ void __launch_bounds__(KV_THREADS, 6)
 kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* __restrict__ k_dst,
                   T* __restrict__ v_dst, KvAddr sa, KvAddr da, int n_kv_heads, int dh, int vis_begin,
-                  int n_text_after, int cap_in, int cap_out, int gather, int rows_per_cta,
+                  int n_text_after, int cap_in, int cap_out, int gather, unsigned magic_ch,
                   const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
                   const int* __restrict__ grp_off, const int* __restrict__ grp_src,
                   const float* __restrict__ weight) {
   constexpr int V = Vec<T>::n;
-  __shared__ int64_t s_src[KV_MAXROWS][KV_MAXM];     // element offset of each member's token
-  __shared__ float s_w[KV_MAXROWS][KV_MAXM];
-  __shared__ int64_t s_dst[KV_MAXROWS];
-  __shared__ int s_cnt[KV_MAXROWS], s_g0[KV_MAXROWS];
-
-  const int b = blockIdx.y, row0 = blockIdx.x * rows_per_cta, tid = threadIdx.x;
+  const int b = blockIdx.y, row = blockIdx.x;
   const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
   const int n_out = n_vis_out[b];
-  const int total_rows = vis_begin + n_out + n_text_after;
-  if (row0 >= total_rows) return;
+  if (row >= vis_begin + n_out + n_text_after) return;
+  const int ch = dh / V, per_kv = n_kv_heads * ch, units = 2 * per_kv;
+  const int64_t d_tok = da.token(b, row);
+  const bool text = row < vis_begin || row >= vis_begin + n_out;
   const int* gs = grp_src + size_t(b) * cap_in;
   const float* wt = weight + size_t(b) * cap_in;
-  const int* go = grp_off + size_t(b) * (cap_out + 1);
-
-  if (tid < rows_per_cta * KV_MAXM) {
-    const int r = tid / KV_MAXM, m = tid - r * KV_MAXM, row = row0 + r;
-    int cnt = 0;
-    if (row < total_rows) {
-      if (row < vis_begin || row >= vis_begin + n_out) {          // text row: copied
-        cnt = 1;
-        if (m == 0) {
-          s_src[r][0] = sa.token(b, row < vis_begin ? row : row - n_out + n_in);
-          s_w[r][0] = 1.0f;
-          s_g0[r] = 0;
-        }
-      } else {
-        const int g0 = go[row - vis_begin];
-        cnt = gather ? 1 : go[row - vis_begin + 1] - g0;
-        if (m < cnt) {
-          const int i = gs[g0 + m];
-          s_src[r][m] = sa.token(b, vis_begin + i);
-          s_w[r][m] = wt[i];
-        }
-        if (m == 0) s_g0[r] = g0;
-      }
-      if (m == 0) s_dst[r] = da.token(b, row);
-    }
-    if (m == 0) s_cnt[r] = cnt;
+  int g0 = 0, g1 = 1;
+  if (!text) {
+    const int* go = grp_off + size_t(b) * (cap_out + 1);
+    g0 = go[row - vis_begin];
+    g1 = gather ? g0 + 1 : go[row - vis_begin + 1];
   }
-  __syncthreads();
-
-  const int ch = dh / V, per_kv = n_kv_heads * ch, units = 2 * per_kv;
-  const int total_items = rows_per_cta * units;
-  for (int base = 0; base < total_items; base += KV_THREADS * KV_ITEMS) {
-    uint4 v[KV_ITEMS][2];
-    int cnt[KV_ITEMS], rr[KV_ITEMS];
-    const T* sp[KV_ITEMS];
-    T* dp[KV_ITEMS];
-#pragma unroll
-    for (int j = 0; j < KV_ITEMS; ++j) {
-      const int idx = base + j * KV_THREADS + tid;
-      cnt[j] = 0;
-      if (idx >= total_items) continue;
-      const int r = idx / units, u = idx - r * units;
-      const int kv = u / per_kv, rem = u - kv * per_kv, h = rem / ch, c = rem - h * ch;
-      rr[j] = r;
-      cnt[j] = s_cnt[r];
-      if (cnt[j] == 0) continue;
-      sp[j] = (kv ? v_src : k_src) + int64_t(h) * sa.head_stride + c * V;
-      dp[j] = (kv ? v_dst : k_dst) + s_dst[r] + int64_t(h) * da.head_stride + c * V;
-      v[j][0] = ld_stream16(sp[j] + s_src[r][0]);
-      if (cnt[j] > 1) v[j][1] = ld_stream16(sp[j] + s_src[r][1]);
+  if (text || g1 - g0 == 1) {                                       // copy: text, lone survivor, gather mode
+    const int64_t s_tok = text ? sa.token(b, row < vis_begin ? row : row - n_out + n_in)
+                               : sa.token(b, vis_begin + gs[g0]);
+    for (int u = threadIdx.x; u < units; u += blockDim.x) {
+      const int kv = u >= per_kv ? 1 : 0, rem = u - kv * per_kv, h = div_magic(rem, magic_ch), c = rem - h * ch;
+      st_stream16((kv ? v_dst : k_dst) + d_tok + int64_t(h) * da.head_stride + c * V,
+                  ld_stream16((kv ? v_src : k_src) + s_tok + int64_t(h) * sa.head_stride + c * V));
     }
+    return;
+  }
+  for (int u = threadIdx.x; u < units; u += blockDim.x) {
+    const int kv = u >= per_kv ? 1 : 0, rem = u - kv * per_kv, h = div_magic(rem, magic_ch), c = rem - h * ch;
+    const T* sp = (kv ? v_src : k_src) + int64_t(h) * sa.head_stride + c * V;
+    float acc[V];
 #pragma unroll
-    for (int j = 0; j < KV_ITEMS; ++j) {
-      if (cnt[j] == 0) continue;
-      if (cnt[j] == 1) { st_stream16(dp[j], v[j][0]); continue; }   // lone survivor / text / gather: copy
-      const int r = rr[j];
-      float acc[V], f[V];
-      unpack16(v[j][0], f, T());
-      const float w0 = s_w[r][0];
+    for (int j = 0; j < V; ++j) acc[j] = 0.f;
+    for (int g = g0; g < g1; g += 4) {                              // up to four members' loads in flight
+      uint4 v[4];
+      float wv[4];
 #pragma unroll
-      for (int e = 0; e < V; ++e) acc[e] = w0 * f[e];
-      unpack16(v[j][1], f, T());
-      const float w1 = s_w[r][1];
-#pragma unroll
-      for (int e = 0; e < V; ++e) acc[e] = fmaf(w1, f[e], acc[e]);
-      for (int m = 2; m < cnt[j]; ++m) {
-        int64_t off;
-        float wv;
-        if (m < KV_MAXM) { off = s_src[r][m]; wv = s_w[r][m]; }
-        else { const int i = gs[s_g0[r] + m]; off = sa.token(b, vis_begin + i); wv = wt[i]; }
-        unpack16(ld_stream16(sp[j] + off), f, T());
-#pragma unroll
-        for (int e = 0; e < V; ++e) acc[e] = fmaf(wv, f[e], acc[e]);
+      for (int m = 0; m < 4; ++m) {
+        if (g + m < g1) {
+          const int i = gs[g + m];
+          wv[m] = wt[i];
+          v[m] = ld_stream16(sp + sa.token(b, vis_begin + i));
+        }
       }
-      st_stream16(dp[j], pack16(acc, T()));
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        if (g + m < g1) {
+          float f[V];
+          unpack16(v[m], f, T());
+#pragma unroll
+          for (int j = 0; j < V; ++j) acc[j] = fmaf(wv[m], f[j], acc[j]);
+        }
+      }
     }
+    st_stream16((kv ? v_dst : k_dst) + d_tok + int64_t(h) * da.head_stride + c * V, pack16(acc, T()));
   }
 }
 
@@ -879,23 +846,24 @@ cudaError_t launch_kv_compact(const KvLaunch& K) {
             a->page_size > 0 ? a->src_block_table : nullptr, a->page_size, a->max_blocks};
   KvAddr da{a->dst_batch_stride, a->dst_head_stride, a->dst_row_stride, a->dst_page_stride,
             a->page_size > 0 ? a->dst_block_table : nullptr, a->page_size, a->max_blocks};
-  const int units = 2 * K.n_kv_heads * (K.head_dim * (K.dtype == LIGHTKV_BF16 ? 2 : 4) / 16);
-  // a CTA resolves the metadata of its tokens once and then moves about KV_BATCHES x 1024 units
-  const int rows_per_cta = std::max(1, std::min(KV_MAXROWS, KV_BATCHES * KV_THREADS * KV_ITEMS / units));
-  const int rows = a->vis_begin + K.cap_out + a->n_text_after;
-  const dim3 grid((rows + rows_per_cta - 1) / rows_per_cta, K.batch);
+  const int ch_host = K.head_dim * (K.dtype == LIGHTKV_BF16 ? 2 : 4) / 16;
+  if (2 * K.n_kv_heads * ch_host >= 65536) return cudaErrorInvalidValue;      // range of the unit decode
+  const unsigned magic_ch = (unsigned)(((1ull << 32) + ch_host - 1) / ch_host);
+  const dim3 grid(a->vis_begin + K.cap_out + a->n_text_after, K.batch);
+  const int units = 2 * K.n_kv_heads * ch_host;
+  const int threads = std::min(KV_THREADS, (units + 31) / 32 * 32);     // narrow caches (GQA) get narrow CTAs
   const int gather = a->mode == LIGHTKV_KV_GATHER;
   if (K.dtype == LIGHTKV_BF16)
-    kv_compact_kernel<__nv_bfloat16><<<grid, KV_THREADS, 0, K.stream>>>(
+    kv_compact_kernel<__nv_bfloat16><<<grid, threads, 0, K.stream>>>(
         static_cast<const __nv_bfloat16*>(a->k_src), static_cast<const __nv_bfloat16*>(a->v_src),
         static_cast<__nv_bfloat16*>(a->k_dst), static_cast<__nv_bfloat16*>(a->v_dst), sa, da, K.n_kv_heads,
-        K.head_dim, a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, rows_per_cta, a->n_vis,
+        K.head_dim, a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, magic_ch, a->n_vis,
         a->n_vis_out, a->grp_off, a->grp_src, a->weight);
   else
-    kv_compact_kernel<float><<<grid, KV_THREADS, 0, K.stream>>>(
+    kv_compact_kernel<float><<<grid, threads, 0, K.stream>>>(
         static_cast<const float*>(a->k_src), static_cast<const float*>(a->v_src),
         static_cast<float*>(a->k_dst), static_cast<float*>(a->v_dst), sa, da, K.n_kv_heads, K.head_dim,
-        a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, rows_per_cta, a->n_vis, a->n_vis_out,
+        a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, magic_ch, a->n_vis, a->n_vis_out,
         a->grp_off, a->grp_src, a->weight);
   return cudaGetLastError();
 }
