@@ -8,7 +8,7 @@ struct LayerLaunch {
   int batch, hidden, n_q_heads, n_kv_heads, head_dim;
   int dtype, xi_mode;
   double keep;
-  int fd_tiles;                      // upper bound on FdTiling::n_tiles of any sample (grid of the tensor-core FD kernel)
+  int fd_tiles;                      // estimate of FdTiling::n_tiles per sample (launch shape of the tensor-core FD kernel)
   Geometry geo;
   Workspace ws;
   const lightkv_layer_args_t* a;

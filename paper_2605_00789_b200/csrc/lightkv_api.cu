@@ -17,7 +17,7 @@ struct StagePlan {
   bool exact;      // cap_in is the exact count (schedule so far is data independent)
   bool exact_out;  // cap_out too
   bool use_tc;
-  int fd_tiles;    // upper bound on the tiles per sample of the tensor-core FD kernel
+  int fd_tiles;    // estimate of the tiles per sample of the tensor-core FD kernel (sizes its launch)
   Geometry geo;
   size_t ws_bytes;
   size_t off[13];     // byte offsets of the Workspace arrays
@@ -36,10 +36,16 @@ namespace lkv {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Upper bound on the tiles per sample the window-build kernel can report when no window has more than
-// max_a A entries: one tile per window while windows fit a tile, else blocks of 128 x 128 per window.
-static int fd_tile_bound(int n_windows, int max_a) {
-  if (max_a <= kFdTile) return n_windows;
+// Tiles per sample the window-build kernel reports when the largest window has max_a A entries (same
+// rule as the kernel).  Only the launch shape of the persistent FD kernel depends on it, so an estimate
+// is enough: the kernel itself walks whatever tiles the device-side tiling holds.
+static int fd_tile_count(int n_windows, int max_a, int batch) {
+  if (max_a <= 0) return 0;
+  if (max_a <= kFdTile) {
+    const int want = (n_windows * batch + kFdTargetTiles - 1) / kFdTargetTiles;
+    const int wpt = std::max(1, std::min(std::min(kFdTile / max_a, n_windows), want));
+    return (n_windows + wpt - 1) / wpt;
+  }
   const int blocks = (max_a + kFdTile - 1) / kFdTile;
   return n_windows * blocks * blocks;
 }
@@ -154,16 +160,18 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
       std::vector<std::vector<int>> members(g.n_windows);
       for (int pos : alive) members[window_of(g, pos)].push_back(pos);   // alive is ascending
       std::vector<int> next;
-      int cap_a = 0, cap_b = 0;
+      int cap_a = 0, cap_b = 0, max_a = 0;
       bool still = true;
       for (const auto& m : members) {
         const int n = (int)m.size(), na = (n + 1) / 2, r = removal_count(n, sp.keep);
         cap_a += na; cap_b += n / 2;
+        max_a = std::max(max_a, na);
         if (r == na && n >= 2) { for (int l = 1; l < n; l += 2) next.push_back(m[l]); }
         else if (r == 0) { next.insert(next.end(), m.begin(), m.end()); }
         else still = false;
       }
       sp.cap_a = cap_a; sp.cap_b = cap_b;
+      sp.fd_tiles = fd_tile_count(g.n_windows, max_a, c->batch);
       if (still) {
         std::sort(next.begin(), next.end());
         alive.swap(next);
@@ -176,13 +184,12 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
       sp.cap_a = (sp.cap_in + sp.n_windows) / 2;
       sp.cap_b = sp.cap_in / 2;
     }
-    {  // Whatever positions the caller passes, a window holds at most the tokens of its grid cell
-       // (balanced cells: ceil(rows/w) x ceil(cols/w)).
+    if (!sp.exact) {  // counts depend on the data: a window holds at most the tokens of its grid cell
+                      // (balanced cells: ceil(rows/w) x ceil(cols/w))
       int cell = 0;
       for (int t = 0; t < c->n_tiles; ++t)
         cell = std::max(cell, ((g.rows[t] + sp.w - 1) / sp.w) * ((g.cols[t] + sp.w - 1) / sp.w));
-      const int max_a = (std::min(cell, sp.cap_in) + 1) / 2;
-      sp.fd_tiles = fd_tile_bound(g.n_windows, max_a);
+      sp.fd_tiles = fd_tile_count(g.n_windows, (std::min(cell, sp.cap_in) + 1) / 2, c->batch);
     }
     if (!exact) {   // data-dependent from here on: every window keeps at most ceil(keep n_w) tokens
       long long bound = (long long)ceil(sp.keep * sp.cap_in) + sp.n_windows;

@@ -282,11 +282,64 @@ struct FdTcArgs {
 constexpr int FT_LOADERS = 256;
 constexpr int FT_STAGES = 6;
 constexpr int FT_AHEAD = 4;                               // fills in flight
+constexpr int kFdPitch = kFdTile + 1;                     // row pitch (floats) of a partial G in shared memory
 constexpr uint32_t FT_STAGE_BYTES = 16 * 1024;
 constexpr uint32_t FT_RING_BYTES = FT_STAGES * FT_STAGE_BYTES + 4096;   // + pad for the 16 KB A read
 constexpr size_t FT_SMEM = size_t(FT_RING_BYTES) + 1024 /* alignment */ + 128 /* barriers */ +
                            4 * kFdTile * sizeof(float);
 
+// Second half of the cluster epilogue (kept out of line so that it does not weigh on the registers of the
+// streaming loop): full norms = partial squared sums added in rank order; then CTA `rank` finishes rows
+// [rank * 128 / ks, (rank + 1) * 128 / ks), a warp per row, lanes over the columns of the row's window.
+__device__ __noinline__ void fd_cluster_finish(const int* a_win, unsigned long long* a_key, int ks, int rank, int a0, int a1,
+                                               int b0, int b1,
+                                               bool combine, const int* win_off, const int* a_off, uint32_t p0,
+                                               const float* a_nrm, const float* b_nrm, float* nrm_a, float* nrm_b,
+                                               volatile int* abort_flag) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  {
+    const int i = tid & (kFdTile - 1);
+    const uint32_t src = smem_u32(tid < kFdTile ? a_nrm + i : b_nrm + i);
+    float ss = 0.f;
+    for (int j = 0; j < ks; ++j) ss += ld_cluster_f32(map_to_cta(src, j));
+    (tid < kFdTile ? nrm_a : nrm_b)[i] = sqrtf(ss);
+  }
+  named_barrier(1, FT_LOADERS);
+  // CTA `rank` finishes rows [rank * 128 / ks, (rank + 1) * 128 / ks): a warp per row, lanes over the
+  // columns of the row's window, partial sums added in rank order
+  const int rows_mine = kFdTile / ks, r0 = rank * rows_mine;
+  for (int rr = warp; rr < rows_mine; rr += 8) {
+    const int row = r0 + rr, e = a0 + row;
+    if (e >= a1) break;                               // warp-uniform; later rows are further out
+    const int w = a_win[e];
+    const int lo = max(win_off[w] - a_off[w], b0) - b0, hi = min(win_off[w + 1] - a_off[w + 1], b1) - b0;
+    const float na = nrm_a[row];
+    float best = 3.0e38f;
+    int best_c = -1;
+    for (int col = lo + lane; col < hi; col += 32) {
+      const uint32_t src = p0 + uint32_t(row * kFdPitch + col) * 4;
+      float gsum = 0.f;
+      for (int j = 0; j < ks; ++j) gsum += ld_cluster_f32(map_to_cta(src, j));
+      const float den = na * nrm_b[col];
+      const float fd = 1.0f - (den > 0.f ? gsum / den : 0.f);
+      if (fd < best) { best = fd; best_c = col; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {                // minimum over the lanes, ties to the lower column
+      const float of = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+      if (oc >= 0 && (best_c < 0 || of < best || (of == best && oc < best_c))) { best = of; best_c = oc; }
+    }
+    if (lane == 0 && best_c >= 0 && !*abort_flag) {
+      const unsigned long long key = ((unsigned long long)orderable(best) << 32) | (unsigned)(b0 + best_c);
+      unsigned long long* dst = a_key + e;
+      if (combine) atomicMin(dst, key); else *dst = key;
+    }
+  }
+}
+
+// CLUSTER = false is the plain launch (ks = 1) with the cluster code compiled out.
+template <bool CLUSTER>
 __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -315,13 +368,17 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t ring = smem_u32(base);
   const int nW = a.ws.n_windows;
-  const int nk = (a.d + 63) >> 6;               // 64-column chunks
+  // A cluster of ks CTAs shares every tile: CTA `rank` contracts chunks [c_lo, c_lo + nk) of the hidden
+  // dimension and the partial results are combined through distributed shared memory (ks = 1: no cluster).
+  const int ks = CLUSTER ? (int)cluster_nctarank() : 1, rank = CLUSTER ? (int)cluster_ctarank() : 0;
+  const int nk_all = (a.d + 63) >> 6;           // 64-column chunks of the whole hidden dimension
+  const int c_lo = rank * nk_all / ks, nk = (rank + 1) * nk_all / ks - c_lo;
 
   // Work items are the (sample, tile) pairs of the whole batch in sample order; this CTA takes items
-  // blockIdx.x, blockIdx.x + gridDim.x, ...  Barrier phases run on across items: `done` counts the
+  // cluster id, cluster id + number of clusters, ...  Barrier phases run on across items: `done` counts the
   // fills this CTA has completed, `n_items` its finished tiles.
   uint32_t done = 0, n_items = 0;
-  for (int item = blockIdx.x;; item += gridDim.x) {
+  for (int item = blockIdx.x / ks;; item += gridDim.x / ks) {
   int b = 0, tile = item;
   while (b < a.batch) {
     const int nt = a.ws.fd_tiling[b].n_tiles;
@@ -348,7 +405,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   if (warp < 8) {
     // ---- gather: thread = 16-byte piece c of row slots g, g + 32, g + 64, g + 96 of every fill
     const int c = tid & 7, g = tid >> 3;
-    const unsigned char* xb = reinterpret_cast<const unsigned char*>(a.x + size_t(b) * a.batch_stride);
+    const unsigned char* xb = reinterpret_cast<const unsigned char*>(a.x + size_t(b) * a.batch_stride) + size_t(c_lo) * 128;
     const int* a_tok = a.ws.a_tok + size_t(b) * a.ws.cap_a;
     const int* b_tok = a.ws.b_tok + size_t(b) * a.ws.cap_b;
     // source row of slot t on even / odd fills (they differ only when passes = 4), validity bits, and the
@@ -385,7 +442,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       for (int t = 0; t < 4; ++t) {
         const int kc = kc0 + (passes == 1 ? (t & 1) : 0);
         if (kc >= nk || !((okm >> t) & 1)) continue;
-        const uint32_t bytes = (kc * 64 + c * 8 < a.d) ? 16u : 0u;   // d is a multiple of 8
+        const uint32_t bytes = ((c_lo + kc) * 64 + c * 8 < a.d) ? 16u : 0u;   // d is a multiple of 8
         const unsigned char* p = odd ? src_o[t] : src_e[t];
         cp_async16(sb + t * 4096, p + (bytes ? size_t(kc0) * 128 : 0), bytes);
       }
@@ -451,7 +508,10 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         ssa[i] += __shfl_xor_sync(0xffffffffu, ssa[i], o);
         ssb[i] += __shfl_xor_sync(0xffffffffu, ssb[i], o);
       }
-      if (c == 0 && i < passes) { a_nrm[g + 32 * i] = sqrtf(ssa[i]); b_nrm[g + 32 * i] = sqrtf(ssb[i]); }
+      if (c == 0 && i < passes) {                         // a cluster exchanges the squared partial sums
+        a_nrm[g + 32 * i] = ks == 1 ? sqrtf(ssa[i]) : ssa[i];
+        b_nrm[g + 32 * i] = ks == 1 ? sqrtf(ssb[i]) : ssb[i];
+      }
     }
     named_barrier(1, FT_LOADERS);
 
@@ -469,7 +529,21 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     const float na = row < cap_rows ? a_nrm[row] : 0.f;
     float best = 3.0e38f;
     int best_c = -1;
-    if (ok) {
+    if (CLUSTER && ok && ks > 1) {
+      // cluster: this CTA's partial G goes to shared memory as float [128][kFdPitch] over the drained ring
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int c0 = half * 64 + j * 32;
+        if (c0 >= n_cols) break;                          // warp-uniform
+        float v[32];
+        tmem_ld32(tmem_base + (uint32_t(q * 32) << 16) + c0, v);
+        tmem_ld_wait();
+        float* prow = reinterpret_cast<float*>(base) + row * kFdPitch + c0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) prow[i] = v[i];
+      }
+    }
+    if (ok && ks == 1) {
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int c0 = half * 64 + j * 32;
@@ -488,6 +562,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         }
       }
     }
+    if (ks == 1) {
     if (half == 1) { red_f[row] = best; red_c[row] = best_c; }
     named_barrier(1, FT_LOADERS);
     if (half == 0 && ok && e < a1) {
@@ -497,6 +572,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         unsigned long long* dst = a.ws.a_key + size_t(b) * a.ws.cap_a + e;
         if (tl.blocks_b > 1) atomicMin(dst, key); else *dst = key;
       }
+    }
     }
     tc_fence_before();                                    // TMEM reads done before the next tile's MMAs
   } else if (lane == 0) {
@@ -535,9 +611,21 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     }
     umma_commit(acc_full);
   }
+  if (CLUSTER && ks > 1) {
+    // ---- cluster epilogue.  Every thread of every CTA of the cluster passes both barriers for every tile,
+    //      whatever happened before (an aborted CTA contributes garbage and the status bit, never a hang).
+    __syncwarp();
+    cluster_sync();                                       // all partial G and squared norms are in shared memory
+    if (warp < 8)
+      fd_cluster_finish(a.ws.a_win + size_t(b) * a.ws.cap_a, a.ws.a_key + size_t(b) * a.ws.cap_a, ks, rank, a0, a1, b0, b1,
+                        tl.blocks_b > 1, win_off, a_off, smem_u32(base), a_nrm, b_nrm, red_f,
+                        reinterpret_cast<float*>(red_c), abort_flag);
+    __syncwarp();
+    cluster_sync();                                       // nobody reads this CTA's shared memory any more
+  }
   done += nf;
   ++n_items;
-  if (*abort_flag) break;
+  if (*abort_flag && ks == 1) break;
   }  // work items
   tc_fence_before();
   __syncthreads();
@@ -569,14 +657,33 @@ cudaError_t launch_fd_tc(const LayerLaunch& L) {
   f.x = static_cast<const __nv_bfloat16*>(a->hidden) + size_t(a->vis_begin) * a->hidden_row_stride;
   f.batch_stride = a->hidden_batch_stride; f.row_stride = a->hidden_row_stride; f.d = L.hidden; f.batch = L.batch;
   f.ws = L.ws; f.status = a->status;
-  cudaError_t e = cudaFuncSetAttribute(fd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM);
-  if (e != cudaSuccess) return e;
-  // persistent CTAs, two per SM, never more than there can be tiles
-  const long long bound = (long long)L.fd_tiles * L.batch;
-  if (bound <= 0) return cudaSuccess;
-  const int grid = (int)std::min<long long>(bound, 2LL * sm_count());
-  fd_tc_kernel<<<grid, FT_LOADERS + 32, FT_SMEM, L.stream>>>(f);
-  return cudaGetLastError();
+  // Persistent CTAs, two per SM, no more than the plan expects tiles.  When that estimate leaves SMs idle,
+  // clusters of 2, 4 or 8 CTAs split the hidden dimension of every tile.
+  const long long bound = std::max<long long>(1, (long long)L.fd_tiles * L.batch);   // an estimate, see the plan
+  const int slots = 2 * sm_count(), nk_all = (L.hidden + 63) / 64;
+  int ks = 1;
+  while (ks < 8 && bound * (2 * ks) <= slots && 2 * ks <= nk_all) ks *= 2;
+  const int clusters = (int)std::min<long long>(bound, slots / ks);
+  cudaError_t e;
+  if (ks == 1) {
+    if ((e = cudaFuncSetAttribute(fd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM)) != cudaSuccess)
+      return e;
+    fd_tc_kernel<false><<<clusters, FT_LOADERS + 32, FT_SMEM, L.stream>>>(f);
+    return cudaGetLastError();
+  }
+  if ((e = cudaFuncSetAttribute(fd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM)) != cudaSuccess)
+    return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(clusters * ks);
+  cfg.blockDim = dim3(FT_LOADERS + 32);
+  cfg.dynamicSmemBytes = FT_SMEM;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = ks; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, fd_tc_kernel<true>, f);
 }
 
 }  // namespace lkv
