@@ -53,6 +53,7 @@ struct Workspace {
   float* xi;       // [B, cap_in]
   int* partner;    // [B, cap_in]         token an A token is merged into, -1 = survives
   int* slot;       // [B, cap_in]         output slot of surviving tokens
+  int* a_partner;  // [B, cap_a]          per A entry: token it is merged into, -1 = survives
   int cap_in, cap_out, cap_a, cap_b, n_windows;
 };
 

@@ -3,6 +3,7 @@
 #include <algorithm>
 
 #include "launch.h"
+#include "tc_common.cuh"
 
 namespace lkv {
 
@@ -463,7 +464,8 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
 }
 
 // =====================================================================================================
-// Selection + merge map (Steps 2-5).  One CTA per sample, phases separated by block barriers.
+// Selection + merge map (Steps 2-5).  One cluster of 1-8 CTAs per sample (about a token per thread), phases
+// separated by cluster barriers, prefix sums across the cluster through distributed shared memory.
 //   0  xi = fixed-order sum over heads (or given / uniform)
 //   1  per window: r = removal_count(n_w); the r A entries with the smallest (FD, index) are selected
 //      (rank by counting; skipped when r = |A|); a selected A token records its best B token
@@ -474,7 +476,6 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
 // =====================================================================================================
 struct SelectArgs {
   int n_q_heads, xi_mode, cap_out;
-  int smem_tokens;                    // tokens the dynamic shared memory has room for (0: use the workspace)
   double keep;
   const int* n_vis;
   const int* pos;
@@ -515,9 +516,15 @@ __device__ inline int block_exclusive_scan(int v, int* warp_sums /* [33] smem */
   return warp_sums[wp] + x - v;
 }
 
+// CLUSTER = false: one CTA per sample, plain launch, block barriers only.
+template <bool CLUSTER>
 __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectArgs a) {
   __shared__ int warp_sums[33];
-  const int b = blockIdx.x, tid = threadIdx.x, nthr = blockDim.x;
+  __shared__ int cta_total[2];                  // survivors / group members counted by this CTA
+  const int cs = CLUSTER ? (int)tc::cluster_nctarank() : 1, rank = CLUSTER ? (int)tc::cluster_ctarank() : 0;
+  auto sync_all = [&]() { if (CLUSTER) tc::cluster_sync(); else __syncthreads(); };
+  const int b = blockIdx.x / cs, tid = threadIdx.x, nthr = blockDim.x;
+  const int gtid = rank * nthr + tid, gthr = cs * nthr;      // thread index / count inside the cluster
   const int nW = ws.n_windows;
   int n = a.n_vis ? min(a.n_vis[b], ws.cap_in) : ws.cap_in;
   if (n < 0) n = 0;
@@ -529,13 +536,10 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   const int* a_win = ws.a_win + size_t(b) * ws.cap_a;
   const unsigned long long* a_key = ws.a_key + size_t(b) * ws.cap_a;
   const int* b_tok = ws.b_tok + size_t(b) * ws.cap_b;
-  // xi, partner and slot are read back through dependent chains in phases 2-5: keep them in shared
-  // memory when the sample fits (the launch passes 12 bytes per token), else in the workspace
-  extern __shared__ __align__(16) unsigned char select_smem[];
-  const bool in_smem = a.smem_tokens >= ws.cap_in;
-  float* xi = in_smem ? reinterpret_cast<float*>(select_smem) : ws.xi + size_t(b) * ws.cap_in;
-  int* partner = in_smem ? reinterpret_cast<int*>(select_smem) + ws.cap_in : ws.partner + size_t(b) * ws.cap_in;
-  int* slot = in_smem ? reinterpret_cast<int*>(select_smem) + 2 * ws.cap_in : ws.slot + size_t(b) * ws.cap_in;
+  float* xi = ws.xi + size_t(b) * ws.cap_in;
+  int* partner = ws.partner + size_t(b) * ws.cap_in;
+  int* slot = ws.slot + size_t(b) * ws.cap_in;
+  int* a_partner = ws.a_partner + size_t(b) * ws.cap_a;
   const int* pos = a.pos ? a.pos + size_t(b) * ws.cap_in : nullptr;
   int* dst = a.dst + size_t(b) * ws.cap_in;
   float* weight = a.weight + size_t(b) * ws.cap_in;
@@ -543,8 +547,42 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   int* grp_src = a.grp_src + size_t(b) * ws.cap_in;
   int* pos_out = a.pos_out + size_t(b) * a.cap_out;
 
+  // Exclusive scan of `value(i)` over i in [0, count) across the whole cluster: every CTA owns a
+  // contiguous range, counts it, learns the ranges before it through distributed shared memory, then
+  // scans its range.  emit(i, prefix) is called for every i; returns the grand total.
+  auto cluster_scan = [&](int count, int which, auto value, auto emit) {
+    const int chunk = (count + cs - 1) / cs, lo = min(count, rank * chunk), hi = min(count, lo + chunk);
+    int before = 0, grand = 0;
+    if (CLUSTER) {
+      int mine = 0;
+      for (int base = lo; base < hi; base += nthr) {
+        const int i = base + tid;
+        int total;
+        block_exclusive_scan(i < hi ? value(i) : 0, warp_sums, &total);
+        mine += total;
+      }
+      if (tid == 0) cta_total[which] = mine;
+      tc::cluster_sync();
+      for (int j = 0; j < cs; ++j) {
+        const int t = (int)tc::ld_cluster_u32(tc::map_to_cta(tc::smem_u32(&cta_total[which]), j));
+        if (j < rank) before += t;
+        grand += t;
+      }
+    }
+    int carry = before;
+    for (int base = lo; base < hi; base += nthr) {
+      const int i = base + tid;
+      const int v = i < hi ? value(i) : 0;
+      int total;
+      const int ex = block_exclusive_scan(v, warp_sums, &total);
+      if (i < hi) emit(i, carry + ex);
+      carry += total;
+    }
+    return CLUSTER ? grand : carry;
+  };
+
   // phase 0
-  for (int i = tid; i < n; i += nthr) {
+  for (int i = gtid; i < n; i += gthr) {
     float v;
     if (a.xi_mode == LIGHTKV_XI_GIVEN) v = a.xi_in[size_t(b) * ws.cap_in + i];
     else if (a.xi_mode == LIGHTKV_XI_UNIFORM) v = 1.0f;
@@ -557,11 +595,11 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     if (a.xi_out) a.xi_out[size_t(b) * ws.cap_in + i] = v;
     partner[i] = -1;
   }
-  __syncthreads();
+  sync_all();
 
   // phase 1
   const int n_a = a_off[nW];
-  for (int e = tid; e < n_a; e += nthr) {
+  for (int e = gtid; e < n_a; e += gthr) {
     const int w = a_win[e];
     const int e_lo = a_off[w], e_hi = a_off[w + 1];
     const int r = removal_count(win_off[w + 1] - win_off[w], a.keep);
@@ -571,37 +609,32 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     else {
       // order by (lowest FD, A entry index): the high word of a_key is the orderable FD
       const unsigned long long key = (a_key[e] & 0xffffffff00000000ull) | (unsigned)e;
-      int rank = 0;
+      int rk = 0;
       for (int e2 = e_lo; e2 < e_hi; ++e2) {
         const unsigned long long k2 = (a_key[e2] & 0xffffffff00000000ull) | (unsigned)e2;
-        rank += (k2 < key);
+        rk += (k2 < key);
       }
-      sel = rank < r;
+      sel = rk < r;
     }
     const unsigned best_e = (unsigned)(a_key[e] & 0xffffffffu);
-    if (sel && best_e != 0xffffffffu) partner[a_tok[e]] = b_tok[best_e];
+    const int p = (sel && best_e != 0xffffffffu) ? b_tok[best_e] : -1;
+    a_partner[e] = p;                                  // entry-indexed copy: the group loops below read it in order
+    if (p >= 0) partner[a_tok[e]] = p;
   }
-  __syncthreads();
+  sync_all();
 
   // phase 2
-  int carry = 0;
-  for (int base = 0; base < n; base += nthr) {
-    const int i = base + tid;
-    const int flag = (i < n && partner[i] < 0) ? 1 : 0;
-    int total;
-    const int ex = block_exclusive_scan(flag, warp_sums, &total);
-    if (flag) slot[i] = carry + ex;
-    carry += total;
-  }
-  const int n_out = min(carry, a.cap_out);
-  if (tid == 0) {
+  const int survivors = cluster_scan(n, 0, [&](int i) { return partner[i] < 0 ? 1 : 0; },
+                                     [&](int i, int prefix) { if (partner[i] < 0) slot[i] = prefix; });
+  const int n_out = min(survivors, a.cap_out);
+  if (gtid == 0) {
     a.n_vis_out[b] = n_out;
-    if (carry > a.cap_out) set_status(a.status, LIGHTKV_STATUS_COUNT);
+    if (survivors > a.cap_out) set_status(a.status, LIGHTKV_STATUS_COUNT);
   }
-  __syncthreads();
+  sync_all();
 
   // phase 3 + 4 (sizes written where the offsets will be)
-  for (int i = tid; i < n; i += nthr) {
+  for (int i = gtid; i < n; i += gthr) {
     const int p = partner[i];
     if (p >= 0) { dst[i] = slot[p]; continue; }
     const int o = slot[i];
@@ -611,25 +644,18 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     int sz = 1;
     if (tok_l[i] & 1) {
       const int w = tok_win[i];
-      for (int e = a_off[w]; e < a_off[w + 1]; ++e) sz += (partner[a_tok[e]] == i);
+      for (int e = a_off[w]; e < a_off[w + 1]; ++e) sz += (a_partner[e] == i);
     }
     grp_off[o] = sz;
   }
-  __syncthreads();
-  carry = 0;
-  for (int base = 0; base < n_out; base += nthr) {
-    const int o = base + tid;
-    const int sz = o < n_out ? grp_off[o] : 0;
-    int total;
-    const int ex = block_exclusive_scan(sz, warp_sums, &total);
-    if (o < n_out) grp_off[o] = carry + ex;
-    carry += total;
-  }
-  if (tid == 0) grp_off[n_out] = carry;
-  __syncthreads();
+  sync_all();
+  const int members = cluster_scan(n_out, 1, [&](int o) { return grp_off[o]; },
+                                   [&](int o, int prefix) { grp_off[o] = prefix; });
+  if (gtid == 0) grp_off[n_out] = members;
+  sync_all();
 
   // phase 5
-  for (int i = tid; i < n; i += nthr) {
+  for (int i = gtid; i < n; i += gthr) {
     if (partner[i] >= 0) continue;
     const int o = slot[i];
     if (o >= a.cap_out) continue;
@@ -640,8 +666,7 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     if (tok_l[i] & 1) {
       const int w = tok_win[i];
       for (int e = a_off[w]; e < a_off[w + 1]; ++e) {
-        const int t = a_tok[e];
-        if (partner[t] == i) { grp_src[off + cnt++] = t; den += xi[t]; }
+        if (a_partner[e] == i) { const int t = a_tok[e]; grp_src[off + cnt++] = t; den += xi[t]; }
       }
     }
     if (den >= 1e-30f) {
@@ -660,14 +685,23 @@ cudaError_t launch_select_map(const LayerLaunch& L) {
   s.n_vis = a->n_vis; s.pos = a->pos; s.xi_in = a->xi; s.n_vis_out = a->n_vis_out; s.pos_out = a->pos_out;
   s.dst = a->dst; s.weight = a->weight; s.grp_off = a->grp_off; s.grp_src = a->grp_src;
   s.xi_out = a->xi_out; s.status = a->status;
-  constexpr int kSelectSmemTokens = 16384;               // 12 bytes per token -> 192 KB
-  const size_t smem = L.ws.cap_in <= kSelectSmemTokens ? size_t(L.ws.cap_in) * 12 : 0;
-  s.smem_tokens = smem ? L.ws.cap_in : 0;
-  cudaError_t e = cudaFuncSetAttribute(select_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kSelectSmemTokens * 12);
-  if (e != cudaSuccess) return e;
-  select_map_kernel<<<L.batch, 1024, smem, L.stream>>>(L.ws, s);
-  return cudaGetLastError();
+  // one cluster per sample: 1, 2, 4 or 8 CTAs of 1024 threads, about one token per thread
+  const int cs = L.ws.cap_in <= 1024 ? 1 : (L.ws.cap_in <= 2048 ? 2 : (L.ws.cap_in <= 4096 ? 4 : 8));
+  if (cs == 1) {
+    select_map_kernel<false><<<L.batch, 1024, 0, L.stream>>>(L.ws, s);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(L.batch * cs);
+  cfg.blockDim = dim3(1024);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = cs; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, select_map_kernel<true>, L.ws, s);
 }
 
 // =====================================================================================================
