@@ -36,9 +36,10 @@ KERNELS = ("window_build", "xi", "fd_best_partner", "select_map", "merge_hidden"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
 # of the stage-0 launch, keyed by (workload, kernel); null where no capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("cfg2", "xi"): 391.76e6,                # profiles/xi_tc_kernel_cfg2_stage0.txt
-    ("cfg2", "fd_best_partner"): 193.17e6,   # profiles/fd_tc_kernel_cfg2_stage0.txt
-    ("cfg2", "merge_hidden"): 264.45e6,      # profiles/merge_rows_kernel_cfg2_stage0.txt
+    ("cfg2", "xi"): 392.01e6,                # profiles/xi_tc_kernel_cfg2_stage0.txt
+    ("cfg2", "fd_best_partner"): 194.49e6,   # profiles/fd_tc_kernel_cfg2_stage0.txt
+    ("cfg2", "merge_hidden"): 264.07e6,      # profiles/merge_rows_kernel_cfg2_stage0.txt
+    ("cfg2", "kv_compact"): 563.58e6,        # profiles/kv_compact_kernel_cfg2_stage0.txt
 }
 
 
@@ -298,11 +299,12 @@ def main():
                           f"keep={list(wl.keep)}, batch {wl.batch}, {wl.n_vis} vision + {wl.n_text} text tokens, "
                           f"hidden {wl.hidden}, {wl.n_q_heads}q/{wl.n_kv_heads}kv heads x {wl.head_dim}, "
                           f"xi from full causal attention, K/V merge, K/V layout {args.kv_layout}",
-              "l2": "inputs larger than L2 (every stage streams > 126 MB)", "batch_per_gpu": wl.batch}
+              "l2": "", "batch_per_gpu": wl.batch}
 
     if args.impl == "reference":
         if rank != 0:
             return
+        config["l2"] = "not applicable (host cores)"
         budget = 150.0
         t_last, tok_last = oracle_sample_step(wl, full_schedule=False)
         full = t_last * 12 * (args.steps + args.warmup) < budget     # the full schedule costs ~10x its last stage
@@ -358,19 +360,39 @@ def main():
         e = torch.cuda.Event(enable_timing=True)
         e.record()                    # torch creates the CUDA event lazily; the C ABI needs a live handle
         return e
+    # A step streams every stage's inputs once.  Where that is less than twice the L2 (small workloads),
+    # the L2 is flushed between timed steps by writing a 256 MB buffer, outside the timed intervals.
+    step_bytes = sum(t.numel() * t.element_size() for s in stages for t in s["host"].values())
+    flush_buf = None
+    if step_bytes < 2 * 126e6:
+        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    config["l2"] = ("L2 flushed between timed steps (256 MB write, untimed)" if flush_buf is not None else
+                    f"inputs larger than L2 ({step_bytes / 1e6:.0f} MB read per step, L2 is 126 MB)")
+
     # timed region: K whole steps in the benchmark's schedule (--streams 2: K/V compaction of a stage on a
-    # second stream, overlapping the next stage's compression)
-    t_begin, t_end = ev(), ev()
+    # second stream, overlapping the next stage's compression).  The clock sampler runs from here to the
+    # end of the per-kernel pass.
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    t_begin.record()
-    for i in range(args.steps):
-        run_step(L, plan, wl, stages, side=side)
-    t_end.record()
-    barrier()
-    clocks = sampler.stop()
-    ms_total = max_over_ranks(t_begin.elapsed_time(t_end), world, device)
+    if flush_buf is None:
+        t_begin, t_end = ev(), ev()
+        t_begin.record()
+        for i in range(args.steps):
+            run_step(L, plan, wl, stages, side=side)
+        t_end.record()
+        barrier()
+        ms_local = t_begin.elapsed_time(t_end)
+    else:
+        pairs = [(ev(), ev()) for _ in range(args.steps)]
+        for a_ev, b_ev in pairs:
+            flush_buf.fill_(1)
+            a_ev.record()
+            run_step(L, plan, wl, stages, side=side)
+            b_ev.record()
+        barrier()
+        ms_local = sum(a_ev.elapsed_time(b_ev) for a_ev, b_ev in pairs)
+    ms_total = max_over_ranks(ms_local, world, device)
     ms_step = ms_total / args.steps
     value = whole_job_throughput(tokens_per_step, world, ms_step)
 
@@ -386,6 +408,7 @@ def main():
         run_step(L, plan, wl, stages, traces[i], kv_ev[i])
     k_end.record()
     barrier()
+    clocks = sampler.stop()
     ms_step_one_stream = max_over_ranks(k_begin.elapsed_time(k_end), world, device) / ksteps
 
     ktime = {k: 0.0 for k in KERNELS}       # ms per step, summed over stages
