@@ -177,12 +177,14 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
           for (int i = 0; i < 32; ++i)
             if (c * 32 + i > lim) v[c][i] = -INFINITY;
       }
-      float mx = v[0][0];
+      float mxc[4];                                     // one dependency chain per 32-column chunk
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
+      for (int c = 0; c < 4; ++c) {
+        mxc[c] = v[c][0];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[c][i]);
-      const float m_new = fmaxf(m_run, mx);
+        for (int i = 1; i < 32; ++i) mxc[c] = fmaxf(mxc[c], v[c][i]);
+      }
+      const float m_new = fmaxf(fmaxf(m_run, fmaxf(mxc[0], mxc[1])), fmaxf(mxc[2], mxc[3]));
       const float ms = m_new * sc;
       float sa = 0.f, st = 0.f;
       if (j0 < a.text_end && j0 + 128 > a.text_begin) {   // tile reaches into the prompt set J
@@ -196,10 +198,12 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
             if (c * 32 + i >= lo && c * 32 + i < hi) st += p;
           }
       } else {
+        float part[4] = {0.f, 0.f, 0.f, 0.f};             // four independent sums
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) sa += ex2(fmaf(v[c][i], sc, -ms));
+          for (int i = 0; i < 32; ++i) part[c] += ex2(fmaf(v[c][i], sc, -ms));
+        sa = (part[0] + part[1]) + (part[2] + part[3]);
       }
       const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
       l_all = fmaf(l_all, resc, sa);
