@@ -173,6 +173,12 @@ typedef struct {
                                       still gets its event).  For per-kernel timing. */
   int32_t seq_rows;                /* rows every (sample, head) slice of q / k really holds (tensor-map
                                       bound of the TMA loads); 0 = vis_begin + cap_in + n_text_after */
+  void*   aux_stream;              /* cudaStream_t or NULL.  When given (and xi comes from Q and K, and no
+                                      trace events are asked for), the window build and the FD kernel, which
+                                      stream the hidden states, are enqueued on this second stream while the
+                                      xi contraction runs on `stream`; the two are forked and joined with
+                                      events inside the call, so the caller sees everything ordered on
+                                      `stream` as before.  The stream must belong to the same device. */
 } lightkv_layer_args_t;
 
 #define LIGHTKV_TRACE_EVENTS 6

@@ -279,16 +279,34 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
 
   cudaEvent_t* ev = reinterpret_cast<cudaEvent_t*>(a->trace_events);
   auto mark = [&](int i) { return ev ? cudaEventRecord(ev[i], L.stream) : cudaSuccess; };
-  if (mark(0) != cudaSuccess) return LIGHTKV_ERR_CUDA;
-  if (launch_window_build(L) != cudaSuccess || mark(1) != cudaSuccess) return LIGHTKV_ERR_CUDA;
-  if (attn) {
-    const bool tc = s.use_tc && c.xi_mode == LIGHTKV_XI_ATTN_FULL && tc_xi_supported(c.head_dim);
-    if ((tc ? launch_xi_tc(L) : launch_xi_simt(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
-  }
-  if (mark(2) != cudaSuccess) return LIGHTKV_ERR_CUDA;
-  {
-    const bool tc = s.use_tc && tc_fd_supported(c.hidden);
-    if ((tc ? launch_fd_tc(L) : launch_fd_simt(L)) != cudaSuccess || mark(3) != cudaSuccess)
+  const bool tc_xi = s.use_tc && c.xi_mode == LIGHTKV_XI_ATTN_FULL && tc_xi_supported(c.head_dim);
+  const bool tc_fd = s.use_tc && tc_fd_supported(c.hidden);
+  cudaStream_t aux = (a->aux_stream && attn && !ev) ? static_cast<cudaStream_t>(a->aux_stream) : nullptr;
+  if (aux) {
+    // fork: window build + FD (HBM bound) on the second stream, xi (bound by the exponentials) on the first
+    cudaEvent_t fork = nullptr, join = nullptr;
+    if (cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&join, cudaEventDisableTiming) != cudaSuccess) {
+      cudaEventDestroy(fork);
+      return LIGHTKV_ERR_CUDA;
+    }
+    LayerLaunch La = L;
+    La.stream = aux;
+    bool ok = cudaEventRecord(fork, L.stream) == cudaSuccess && cudaStreamWaitEvent(aux, fork, 0) == cudaSuccess;
+    ok = ok && launch_window_build(La) == cudaSuccess;
+    ok = ok && (tc_fd ? launch_fd_tc(La) : launch_fd_simt(La)) == cudaSuccess;
+    ok = ok && cudaEventRecord(join, aux) == cudaSuccess;
+    ok = ok && (tc_xi ? launch_xi_tc(L) : launch_xi_simt(L)) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(L.stream, join, 0) == cudaSuccess;
+    cudaEventDestroy(fork);                 // released once the recorded work has completed
+    cudaEventDestroy(join);
+    if (!ok) return LIGHTKV_ERR_CUDA;
+  } else {
+    if (mark(0) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    if (launch_window_build(L) != cudaSuccess || mark(1) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    if (attn && (tc_xi ? launch_xi_tc(L) : launch_xi_simt(L)) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    if (mark(2) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    if ((tc_fd ? launch_fd_tc(L) : launch_fd_simt(L)) != cudaSuccess || mark(3) != cudaSuccess)
       return LIGHTKV_ERR_CUDA;
   }
   if (launch_select_map(L) != cudaSuccess || mark(4) != cudaSuccess) return LIGHTKV_ERR_CUDA;

@@ -77,7 +77,7 @@ def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_t
 
 
 def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0, text_range=None,
-              lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None):
+              lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None, aux_stream=None):
     """Run lightkv_compress_layer (or `layer_fn`, a binding function with the same signature) +
     lightkv_compact_kv on the device; returns numpy outputs."""
     import torch
@@ -89,6 +89,8 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
     n_seq = hidden.shape[1]
     assert n_seq <= vb + info.cap_in + n_text_after
     kw = {}
+    if aux_stream is not None:
+        kw["aux_stream"] = aux_stream
     if xi_mode in ("attn", "lse"):
         kw["q"], kw["k"] = to_device(inp["q"], dtype, device), to_device(inp["k"], dtype, device)
     if xi_mode == "lse":
@@ -211,7 +213,7 @@ def compare_stage(wl, stage, inp, ref, gpu, dtype="bf16", kv_mode="merge", n_tex
 
 
 def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge", paged=0, samples=None,
-                 stages=None, oracle_samples=None):
+                 stages=None, oracle_samples=None, aux_stream=None):
     """All stages of a workload, chained through the surviving positions; returns per-stage stats."""
     bsz = wl.batch if samples is None else len(samples)
     plan = make_plan(wl, dtype, xi_mode, engine, batch=bsz)
@@ -223,7 +225,8 @@ def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge
             rng = np.random.default_rng(stage)
             inp["xi"] = rng.uniform(0.05, 3.0, size=inp["pos"].shape).astype(np.float32)
         lse = oracle_lse(inp, wl.n_q_heads, wl.n_kv_heads) if xi_mode == "lse" else None
-        gpu = gpu_stage(plan, wl, stage, inp, dtype, xi_mode, lse=lse, kv_mode=kv_mode, paged=paged)
+        gpu = gpu_stage(plan, wl, stage, inp, dtype, xi_mode, lse=lse, kv_mode=kv_mode, paged=paged,
+                        aux_stream=aux_stream)
         osamp = list(range(bsz)) if oracle_samples is None else oracle_samples
         sub = {key: (val[osamp] if isinstance(val, np.ndarray) and val.shape[:1] == (bsz,) else val)
                for key, val in inp.items()}

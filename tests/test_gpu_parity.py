@@ -56,6 +56,15 @@ def test_cfg1_full_schedule(name):
         assert [s["n_out"] for s in stats] == [[288], [144], [72]]
 
 
+@pytest.mark.parametrize("name", ["small", "cfg1"])
+def test_second_stream_inside_compress_layer(name):
+    # window build + FD on aux_stream beside xi: same results as the oracle, run after run
+    import torch
+    aux = torch.cuda.Stream()
+    for _ in range(2):
+        H.run_schedule(S.workload(name), aux_stream=aux)
+
+
 def test_cfg0_fp32_mode():
     H.run_schedule(dataclasses.replace(S.workload("cfg0"), hidden=1024, n_q_heads=8, n_kv_heads=8), dtype="fp32")
 
