@@ -462,17 +462,38 @@ def main():
         h2d = sum(t.numel() * t.element_size() for s in stages for t in s["host"].values())
         d2h = sum(t.numel() * t.element_size() for s in stages for t in s["host_out"].values())
 
+        cin, cout = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
+        kv_side = side if side is not None else torch.cuda.current_stream()
+
         def e2e_step():
+            """One step from pinned host inputs to pinned host outputs: every stage's inputs go up on a copy
+            stream while earlier stages compute, results come down on another as soon as they exist."""
+            main = torch.cuda.current_stream()
+            cin.wait_stream(main)                       # the previous step no longer reads the device inputs
+            ready = []
+            with torch.cuda.stream(cin):
+                for s in stages:
+                    for name, t in s["host"].items():
+                        s["dev"][name].copy_(t, non_blocking=True)
+                    e = torch.cuda.Event()
+                    e.record(cin)
+                    ready.append(e)
+            pos, n_vis = stages[0]["dev"]["pos"], stages[0]["dev"]["n_vis"]
             for st, s in enumerate(stages):
-                for name, t in s["host"].items():
-                    s["dev"][name].copy_(t, non_blocking=True)
-            run_step(L, plan, wl, stages, side=side, aux=aux)
-            for s in stages:
-                s["host_out"]["hidden"].copy_(s["out"].hidden_out, non_blocking=True)
-                s["host_out"]["k"].copy_(s["k_dst"], non_blocking=True)
-                s["host_out"]["v"].copy_(s["v_dst"], non_blocking=True)
-                s["host_out"]["n_vis_out"].copy_(s["out"].n_vis_out, non_blocking=True)
-                s["host_out"]["pos_out"].copy_(s["out"].pos_out, non_blocking=True)
+                main.wait_event(ready[st])
+                run_stage(L, plan, wl, st, s, pos, n_vis, side=side, aux=aux)
+                cout.wait_stream(main)
+                cout.wait_stream(kv_side)
+                with torch.cuda.stream(cout):
+                    s["host_out"]["hidden"].copy_(s["out"].hidden_out, non_blocking=True)
+                    s["host_out"]["k"].copy_(s["k_dst"], non_blocking=True)
+                    s["host_out"]["v"].copy_(s["v_dst"], non_blocking=True)
+                    s["host_out"]["n_vis_out"].copy_(s["out"].n_vis_out, non_blocking=True)
+                    s["host_out"]["pos_out"].copy_(s["out"].pos_out, non_blocking=True)
+                pos, n_vis = s["out"].pos_out, s["out"].n_vis_out
+            if side is not None:
+                main.wait_stream(side)
+            main.wait_stream(cout)
         e2e_steps = max(3, min(args.steps, 10))
         for _ in range(2):
             e2e_step()

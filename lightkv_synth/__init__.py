@@ -36,7 +36,7 @@ TENSOR_HIDDEN, TENSOR_Q, TENSOR_K, TENSOR_V = 0, 1, 2, 3
 
 @dataclasses.dataclass(frozen=True)
 class Workload:
-    """Shape and schedule of one synthetic workload (one BASELINE config)."""
+    """Shape and schedule of one synthetic workload."""
     name: str
     config_id: int
     batch: int

@@ -77,7 +77,8 @@ def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_t
 
 
 def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0, text_range=None,
-              lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None, aux_stream=None):
+              lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None, aux_stream=None,
+              kv_layout="bhnd"):
     """Run lightkv_compress_layer (or `layer_fn`, a binding function with the same signature) +
     lightkv_compact_kv on the device; returns numpy outputs."""
     import torch
@@ -142,6 +143,10 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
         else:
             k_dst = torch.full((bsz, hkv, n_seq_out, dh), float("nan"), dtype=tdt, device=device)
             v_dst = k_dst.clone()
+            if kv_layout == "bnhd":      # token-major storage [B, N, H_kv, dh] handed over as strided views
+                as_bnhd = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+                k_src, v_src, k_dst, v_dst = as_bnhd(k_src), as_bnhd(v_src), as_bnhd(k_dst), as_bnhd(v_dst)
+                assert k_src.stride(1) == dh and k_src.stride(2) == hkv * dh
             L.compact_kv(plan, stage, out, k_src, v_src, k_dst, v_dst, vis_begin=vb, n_text_after=n_text_after,
                          mode=mode, n_vis=torch.from_numpy(inp["n_vis"]).to(device))
         torch.cuda.synchronize()
@@ -213,7 +218,7 @@ def compare_stage(wl, stage, inp, ref, gpu, dtype="bf16", kv_mode="merge", n_tex
 
 
 def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge", paged=0, samples=None,
-                 stages=None, oracle_samples=None, aux_stream=None):
+                 stages=None, oracle_samples=None, aux_stream=None, kv_layout="bhnd"):
     """All stages of a workload, chained through the surviving positions; returns per-stage stats."""
     bsz = wl.batch if samples is None else len(samples)
     plan = make_plan(wl, dtype, xi_mode, engine, batch=bsz)
@@ -226,7 +231,7 @@ def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge
             inp["xi"] = rng.uniform(0.05, 3.0, size=inp["pos"].shape).astype(np.float32)
         lse = oracle_lse(inp, wl.n_q_heads, wl.n_kv_heads) if xi_mode == "lse" else None
         gpu = gpu_stage(plan, wl, stage, inp, dtype, xi_mode, lse=lse, kv_mode=kv_mode, paged=paged,
-                        aux_stream=aux_stream)
+                        aux_stream=aux_stream, kv_layout=kv_layout)
         osamp = list(range(bsz)) if oracle_samples is None else oracle_samples
         sub = {key: (val[osamp] if isinstance(val, np.ndarray) and val.shape[:1] == (bsz,) else val)
                for key, val in inp.items()}

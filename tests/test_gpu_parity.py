@@ -41,6 +41,12 @@ def test_small_kv_modes_and_paged_cache(kv_mode, paged):
     H.run_schedule(S.workload("small"), kv_mode=kv_mode, paged=paged, stages=[0])
 
 
+@pytest.mark.parametrize("kv_mode", ["merge", "gather"])
+def test_small_token_major_kv_cache(kv_mode):
+    # K/V stored [B, N, H_kv, dh]: the same call with other strides
+    H.run_schedule(S.workload("small"), kv_mode=kv_mode, kv_layout="bnhd", stages=[0, 1])
+
+
 @pytest.mark.parametrize("w", [4, 6, 1])
 @pytest.mark.parametrize("engine", ["simt", "auto"])
 def test_cfg0_single_step(w, engine):
