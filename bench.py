@@ -128,7 +128,21 @@ def whole_job_throughput(tokens_per_rank_step: int, world: int, ms_step_max: flo
 
 # ------------------------------------------------------------------------------------------ workload
 
-def build_inputs(wl, plan, L, torch, device, sample_offset, kv_layout="bhnd"):
+def causal_lse(torch, q, k, group):
+    """Row log-sum-exp of the scaled causal logits, [B, H, N] fp32 (what a fused attention kernel hands over);
+    plain torch, one sample at a time: an input of the lse mode, computed outside every timed region."""
+    b, h, n, dh = q.shape
+    out = torch.empty((b, h, n), dtype=torch.float32, device=q.device)
+    mask = torch.ones((n, n), dtype=torch.bool, device=q.device).tril_()
+    for i in range(b):
+        kk = k[i].float().repeat_interleave(group, dim=0)
+        for h0 in range(0, h, 8):
+            logits = torch.matmul(q[i, h0:h0 + 8].float(), kk[h0:h0 + 8].transpose(1, 2)) / dh ** 0.5
+            out[i, h0:h0 + 8] = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
+    return out
+
+
+def build_inputs(wl, plan, L, torch, device, sample_offset, kv_layout="bhnd", xi_mode="full"):
     """Generate every stage's inputs on the host (pinned) and upload them.  Stage i+1 is sampled at the
     positions that survive stage i (taken from one untimed run of the library itself)."""
     samples = rank_samples(sample_offset // wl.batch, wl.batch)
@@ -149,6 +163,8 @@ def build_inputs(wl, plan, L, torch, device, sample_offset, kv_layout="bhnd"):
         n_seq = host["hidden"].shape[1]
         pos_pad = np.full((wl.batch, info.cap_in), -1, dtype=np.int32)
         pos_pad[:, :inp["pos"].shape[1]] = inp["pos"]
+        if xi_mode == "lse":
+            dev["lse"] = causal_lse(torch, dev["q"], dev["k"], wl.n_q_heads // wl.n_kv_heads)
         dev["pos"] = torch.from_numpy(pos_pad).to(device)
         dev["n_vis"] = torch.from_numpy(inp["n_vis"]).to(device)
         n_seq_out = wl.n_text + info.cap_out
@@ -186,7 +202,7 @@ def run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None, side=None, aux=None)
     import torch
     d = stg["dev"]
     L.compress_layer(plan, st, d["hidden"], stg["out"], vis_begin=wl.n_text, q=d["q"], k=d["k"], n_vis=n_vis,
-                     pos=pos, trace_events=trace, aux_stream=aux)
+                     pos=pos, trace_events=trace, aux_stream=aux, lse=d.get("lse"))
     if side is None:
         L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
                      n_vis=n_vis)
@@ -212,7 +228,7 @@ def run_step(L, plan, wl, stages, traces=None, kv_events=None, side=None, aux=No
         torch.cuda.current_stream().wait_stream(side)
 
 
-def algorithmic_work(wl, stages):
+def algorithmic_work(wl, stages, xi_mode="full"):
     """Per stage and per kernel: algorithmic bytes (HBM streams) or flops (xi) of one launch."""
     e = 2  # bf16
     per_stage = []
@@ -223,6 +239,8 @@ def algorithmic_work(wl, stages):
         n_out = stg["n_out"].astype(np.float64)
         # xi, ATTN_FULL: 2*dh flops per (head, query, visible key); query t sees n_text + t + 1 keys
         work["xi"] = float((2.0 * wl.n_q_heads * wl.head_dim * (n_in * (nt + 1) + n_in * (n_in - 1) / 2)).sum())
+        if xi_mode == "lse":       # only the prompt keys: 2*dh flops per (head, query, prompt key)
+            work["xi"] = float((2.0 * wl.n_q_heads * wl.head_dim * n_in * nt).sum())
         # FD: one read of the vision rows (+ 8 bytes of keys per A node)
         work["fd_best_partner"] = float((n_in * wl.hidden * e + 4 * n_in).sum())
         # hidden merge: every input row read once, every output row written once
@@ -282,6 +300,9 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(S.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--engine", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--xi-mode", default="full", choices=["full", "lse"],
+                    help="full: xi from Q and K alone (the benchmark); lse: the row log-sum-exp of the layer's attention "
+                         "is an input (computed once with torch before the timed region), only prompt keys are visited")
     ap.add_argument("--kv-layout", default="bhnd", choices=["bhnd", "bnhd"],
                     help="K/V cache layout: [B,H_kv,N,dh] (head-major) or [B,N,H_kv,dh] (token-major)")
     ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
@@ -299,7 +320,8 @@ def main():
     config = {"workload": f"{wl.name}: {wl.n_stages}-stage schedule layers={list(wl.layers)} windows={list(wl.windows)} "
                           f"keep={list(wl.keep)}, batch {wl.batch}, {wl.n_vis} vision + {wl.n_text} text tokens, "
                           f"hidden {wl.hidden}, {wl.n_q_heads}q/{wl.n_kv_heads}kv heads x {wl.head_dim}, "
-                          f"xi from full causal attention, K/V merge, K/V layout {args.kv_layout}",
+                          f"xi from {'full causal attention' if args.xi_mode == 'full' else 'the prompt keys + a given row log-sum-exp'}, "
+                          f"K/V merge, K/V layout {args.kv_layout}",
               "l2": "", "batch_per_gpu": wl.batch}
 
     if args.impl == "reference":
@@ -342,9 +364,11 @@ def main():
     import paper_2605_00789_b200 as L
 
     plan = L.Plan(wl.batch, wl.hidden, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_layers, wl.tiles, wl.layers,
-                  wl.windows, wl.keep, wl.n_text, dtype=L.BF16, xi_mode=L.XI_ATTN_FULL,
+                  wl.windows, wl.keep, wl.n_text, dtype=L.BF16,
+                  xi_mode=L.XI_ATTN_FULL if args.xi_mode == "full" else L.XI_ATTN_LSE,
                   engine=L.ENGINE_AUTO if args.engine == "auto" else L.ENGINE_SIMT)
-    stages = build_inputs(wl, plan, L, torch, device, sample_offset=rank * wl.batch, kv_layout=args.kv_layout)
+    stages = build_inputs(wl, plan, L, torch, device, sample_offset=rank * wl.batch, kv_layout=args.kv_layout,
+                          xi_mode=args.xi_mode)
     tokens_per_step = int(sum(int(s["n_vis"].sum()) for s in stages))
     n_stages = len(stages)
 
@@ -424,7 +448,7 @@ def main():
     for st in range(n_stages):
         for k in KERNELS:
             ktime[k] += kstage[st][k]
-    work_stage = algorithmic_work(wl, stages)
+    work_stage = algorithmic_work(wl, stages, args.xi_mode)
     work = {k: sum(w[k] for w in work_stage) for k in KERNELS}
     peaks = measured_peaks()
 

@@ -216,7 +216,8 @@ int lightkv_plan_stage_info(const lightkv_plan_t* p, int32_t stage, lightkv_stag
   info->cap_in = s.cap_in; info->cap_out = s.cap_out; info->n_windows = s.n_windows;
   info->counts_exact = (s.exact && s.exact_out) ? 1 : 0;
   info->uses_tensor_cores = (s.use_tc && (tc_fd_supported(p->cfg.hidden) ||
-                                          ((p->cfg.xi_mode == LIGHTKV_XI_ATTN_FULL) &&
+                                          ((p->cfg.xi_mode == LIGHTKV_XI_ATTN_FULL ||
+                                            p->cfg.xi_mode == LIGHTKV_XI_ATTN_LSE) &&
                                            tc_xi_supported(p->cfg.head_dim)))) ? 1 : 0;
   info->workspace_bytes = s.ws_bytes;
   return LIGHTKV_OK;
@@ -279,7 +280,7 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
 
   cudaEvent_t* ev = reinterpret_cast<cudaEvent_t*>(a->trace_events);
   auto mark = [&](int i) { return ev ? cudaEventRecord(ev[i], L.stream) : cudaSuccess; };
-  const bool tc_xi = s.use_tc && c.xi_mode == LIGHTKV_XI_ATTN_FULL && tc_xi_supported(c.head_dim);
+  const bool tc_xi = s.use_tc && attn && tc_xi_supported(c.head_dim);
   const bool tc_fd = s.use_tc && tc_fd_supported(c.hidden);
   cudaStream_t aux = (a->aux_stream && attn && !ev) ? static_cast<cudaStream_t>(a->aux_stream) : nullptr;
   if (aux) {

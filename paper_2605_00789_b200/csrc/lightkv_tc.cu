@@ -66,6 +66,8 @@ struct XiTcArgs {
   const int* n_vis;
   float* xi_h;
   uint32_t* status;
+  const float* lse;                  // [B, H, N] row log-sum-exp (natural log) from the caller, or nullptr
+  int64_t lse_bs, lse_hs;
   int cap_in, vis_begin, text_begin, text_end, n_q_heads, group;
   float scale2;                      // log2(e) / sqrt(dh)
 };
@@ -97,7 +99,10 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   if (t0 >= n) return;
   const int nq = min(128, n - t0);
   const int s_first = a.vis_begin + t0, s_last = s_first + nq - 1;
-  const int nkt = s_last / 128 + 1;
+  // key tiles to visit: all tiles up to the last query's own key, or, when the caller supplies the row
+  // log-sum-exp, only the tiles that hold prompt keys (J lies before the vision block, so it is visible)
+  const int kt_lo = a.lse ? a.text_begin / 128 : 0;
+  const int nkt = a.lse ? (a.text_end > a.text_begin ? (a.text_end - 1) / 128 + 1 - kt_lo : 0) : s_last / 128 + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -127,7 +132,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         mbar_expect_tx(&k_full[s], TILE_BYTES);
 #pragma unroll
         for (int hf = 0; hf < HALVES; ++hf)
-          tma_load_4d(k_s + s * TILE_BYTES + hf * 16384, &k_map, &k_full[s], hf * 64, kt * 128, hk, b);
+          tma_load_4d(k_s + s * TILE_BYTES + hf * 16384, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * 128, hk, b);
       }
     }
   } else if (warp == 1) {
@@ -157,7 +162,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
     const float sc = a.scale2;
     for (int kt = 0; kt < nkt; ++kt) {
-      const int buf = kt & 1, j0 = kt * 128;
+      const int buf = kt & 1, j0 = (kt_lo + kt) * 128;
       const bool landed = mbar_wait(&s_full[buf], (kt >> 1) & 1, abort_flag);
       if (!__all_sync(0xffffffffu, landed)) break;        // the TMEM loads below are warp-wide
       tc_fence_after();
@@ -169,6 +174,19 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_empty[buf]);
 
+      if (a.lse) {                                      // normaliser known: only the prompt columns count
+        const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
+        const int lo = a.text_begin - j0, hi = a.text_end - j0;
+        float st = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c * 32 + i >= lo && c * 32 + i < hi) st += ex2(fmaf(v[c][i], sc, -l2));
+        l_txt += st;
+        l_all = 1.f;
+        continue;
+      }
       if (j0 + 127 > s_first) {                         // tile straddles the diagonal: causal mask
         const int lim = s_first + r - j0;               // last visible column of this row
 #pragma unroll
@@ -211,7 +229,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       m_run = m_new;
     }
     if (r < nq && !*abort_flag)
-      a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + t0 + r] = l_txt / l_all;
+      a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + t0 + r] = a.lse ? l_txt : l_txt / l_all;
   }
   tc_fence_before();
   __syncthreads();
@@ -235,6 +253,7 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
     return cudaErrorInvalidValue;
   XiTcArgs x;
   x.n_vis = a->n_vis; x.xi_h = L.ws.xi_h; x.status = a->status; x.cap_in = L.ws.cap_in;
+  x.lse = L.xi_mode == LIGHTKV_XI_ATTN_LSE ? a->lse : nullptr; x.lse_bs = a->lse_batch_stride; x.lse_hs = a->lse_head_stride;
   x.vis_begin = a->vis_begin; x.text_begin = a->text_begin; x.text_end = a->text_end;
   x.n_q_heads = L.n_q_heads; x.group = L.n_q_heads / L.n_kv_heads;
   x.scale2 = 1.4426950408889634f / sqrtf((float)L.head_dim);

@@ -41,6 +41,13 @@ def test_small_kv_modes_and_paged_cache(kv_mode, paged):
     H.run_schedule(S.workload("small"), kv_mode=kv_mode, paged=paged, stages=[0])
 
 
+def test_small_lse_mode_on_tensor_cores():
+    # row log-sum-exp supplied by the caller: only the prompt key tiles are visited (tcgen05 path, GQA)
+    H.run_schedule(S.workload("small"), xi_mode="lse")
+    wl = dataclasses.replace(S.workload("cfg0"), n_text=200)      # prompt keys spanning two key tiles
+    H.run_schedule(wl, xi_mode="lse")
+
+
 @pytest.mark.parametrize("kv_mode", ["merge", "gather"])
 def test_small_token_major_kv_cache(kv_mode):
     # K/V stored [B, N, H_kv, dh]: the same call with other strides
