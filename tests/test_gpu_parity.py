@@ -157,12 +157,16 @@ def test_cfg2_full_size_sampled():
     assert [s["n_out"] for s in stats] == [[1440] * 8, [720] * 8, [360] * 8]
 
 
-def test_cfg3_first_stage_sampled():
-    H.run_schedule(S.workload("cfg3"), stages=[0], oracle_samples=[0, 31])
+def test_cfg3_full_schedule_sampled():
+    stats = H.run_schedule(S.workload("cfg3"), oracle_samples=[0, 31])
+    assert [s["n_out"] for s in stats] == [[288] * 32, [144] * 32, [72] * 32]
 
 
-def test_cfg4_gqa_video_first_stage_sampled():
-    H.run_schedule(S.workload("cfg4"), stages=[0], oracle_samples=[1])
+def test_cfg4_gqa_video_full_schedule_sampled():
+    # all three stages: later stages have few large tiles (128 x 128 entries), which the FD kernel splits
+    # over clusters of CTAs, and 8192 -> 2048 tokens per sample for the clustered selection kernel
+    stats = H.run_schedule(S.workload("cfg4"), oracle_samples=[1])
+    assert [s["n_out"] for s in stats] == [[4096] * 2, [2048] * 2, [1024] * 2]
 
 
 def test_cfg4g_large_windows_uniform_xi():
