@@ -73,17 +73,21 @@ struct XiTcArgs {
 };
 
 constexpr int XT_STAGES = 2;
+constexpr int XT_KEY_TILE = 64;      // keys per tile (64: three CTAs per SM; 128: two)
 
-template <int DH>
-__global__ void __launch_bounds__(192, 2)
+template <int DH, int BK>
+__global__ void __launch_bounds__(192, BK == 64 ? 3 : 2)
 xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, XiTcArgs a) {
   constexpr int HALVES = DH / 64;
-  constexpr uint32_t TILE_BYTES = HALVES * 16384;          // 128 rows x DH bf16
+  constexpr uint32_t TILE_BYTES = HALVES * 16384;          // Q tile: 128 rows x DH bf16
+  constexpr uint32_t KHALF_BYTES = BK * 128;               // BK key rows x 64 columns
+  constexpr uint32_t KT_BYTES = HALVES * KHALF_BYTES;      // K tile: BK rows x DH bf16
+  constexpr int NC = BK / 32;                              // 32-column chunks of a tile
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* q_s = base;
   unsigned char* k_s = base + TILE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(base + TILE_BYTES * (1 + XT_STAGES));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + TILE_BYTES + KT_BYTES * XT_STAGES);
   uint64_t* q_full = bars;
   uint64_t* k_full = bars + 1;                 // [XT_STAGES]
   uint64_t* k_empty = k_full + XT_STAGES;      // [XT_STAGES]
@@ -101,8 +105,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   const int s_first = a.vis_begin + t0, s_last = s_first + nq - 1;
   // key tiles to visit: all tiles up to the last query's own key, or, when the caller supplies the row
   // log-sum-exp, only the tiles that hold prompt keys (J lies before the vision block, so it is visible)
-  const int kt_lo = a.lse ? a.text_begin / 128 : 0;
-  const int nkt = a.lse ? (a.text_end > a.text_begin ? (a.text_end - 1) / 128 + 1 - kt_lo : 0) : s_last / 128 + 1;
+  const int kt_lo = a.lse ? a.text_begin / BK : 0;
+  const int nkt = a.lse ? (a.text_end > a.text_begin ? (a.text_end - 1) / BK + 1 - kt_lo : 0) : s_last / BK + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -112,7 +116,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     *abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, 256); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(tmem_slot, 2 * BK); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -129,15 +133,15 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       for (int kt = 0; kt < nkt; ++kt) {
         const int s = kt % XT_STAGES;
         if (!mbar_wait(&k_empty[s], ((kt / XT_STAGES) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(&k_full[s], TILE_BYTES);
+        mbar_expect_tx(&k_full[s], KT_BYTES);
 #pragma unroll
         for (int hf = 0; hf < HALVES; ++hf)
-          tma_load_4d(k_s + s * TILE_BYTES + hf * 16384, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * 128, hk, b);
+          tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, b);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(128, 128);
+      constexpr uint32_t idesc = idesc_bf16(128, BK);
       const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s);
       bool ok = mbar_wait(q_full, 0, abort_flag);
       for (int kt = 0; ok && kt < nkt; ++kt) {
@@ -147,9 +151,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-          umma_bf16(tmem_base + buf * 128, smem_desc_sw128(q_addr + off),
-                    smem_desc_sw128(k_addr + s * TILE_BYTES + off), idesc, kk > 0);
+          umma_bf16(tmem_base + buf * BK, smem_desc_sw128(q_addr + (kk >> 2) * 16384 + (kk & 3) * 32),
+                    smem_desc_sw128(k_addr + s * KT_BYTES + (kk >> 2) * KHALF_BYTES + (kk & 3) * 32), idesc, kk > 0);
         }
         umma_commit(&k_empty[s]);
         umma_commit(&s_full[buf]);
@@ -162,13 +165,13 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
     const float sc = a.scale2;
     for (int kt = 0; kt < nkt; ++kt) {
-      const int buf = kt & 1, j0 = (kt_lo + kt) * 128;
+      const int buf = kt & 1, j0 = (kt_lo + kt) * BK;
       const bool landed = mbar_wait(&s_full[buf], (kt >> 1) & 1, abort_flag);
       if (!__all_sync(0xffffffffu, landed)) break;        // the TMEM loads below are warp-wide
       tc_fence_after();
-      float v[4][32];
+      float v[NC][32];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(lane_addr + buf * 128 + c * 32, v[c]);
+      for (int c = 0; c < NC; ++c) tmem_ld32(lane_addr + buf * BK + c * 32, v[c]);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
@@ -179,7 +182,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         const int lo = a.text_begin - j0, hi = a.text_end - j0;
         float st = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < NC; ++c)
 #pragma unroll
           for (int i = 0; i < 32; ++i)
             if (c * 32 + i >= lo && c * 32 + i < hi) st += ex2(fmaf(v[c][i], sc, -l2));
@@ -187,28 +190,30 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         l_all = 1.f;
         continue;
       }
-      if (j0 + 127 > s_first) {                         // tile straddles the diagonal: causal mask
+      if (j0 + BK - 1 > s_first) {                         // tile straddles the diagonal: causal mask
         const int lim = s_first + r - j0;               // last visible column of this row
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < NC; ++c)
 #pragma unroll
           for (int i = 0; i < 32; ++i)
             if (c * 32 + i > lim) v[c][i] = -INFINITY;
       }
-      float mxc[4];                                     // one dependency chain per 32-column chunk
+      float mxc[NC];                                     // one dependency chain per 32-column chunk
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < NC; ++c) {
         mxc[c] = v[c][0];
 #pragma unroll
         for (int i = 1; i < 32; ++i) mxc[c] = fmaxf(mxc[c], v[c][i]);
       }
-      const float m_new = fmaxf(fmaxf(m_run, fmaxf(mxc[0], mxc[1])), fmaxf(mxc[2], mxc[3]));
+      float m_new = m_run;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) m_new = fmaxf(m_new, mxc[c]);
       const float ms = m_new * sc;
       float sa = 0.f, st = 0.f;
-      if (j0 < a.text_end && j0 + 128 > a.text_begin) {   // tile reaches into the prompt set J
+      if (j0 < a.text_end && j0 + BK > a.text_begin) {   // tile reaches into the prompt set J
         const int lo = a.text_begin - j0, hi = a.text_end - j0;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < NC; ++c)
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const float p = ex2(fmaf(v[c][i], sc, -ms));
@@ -216,12 +221,15 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
             if (c * 32 + i >= lo && c * 32 + i < hi) st += p;
           }
       } else {
-        float part[4] = {0.f, 0.f, 0.f, 0.f};             // four independent sums
+        float part[NC];                                   // independent sums
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < NC; ++c) part[c] = 0.f;
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
 #pragma unroll
           for (int i = 0; i < 32; ++i) part[c] += ex2(fmaf(v[c][i], sc, -ms));
-        sa = (part[0] + part[1]) + (part[2] + part[3]);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) sa += part[c];
       }
       const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
       l_all = fmaf(l_all, resc, sa);
@@ -235,7 +243,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 256);
+    tmem_dealloc(tmem_base, 2 * BK);
   }
   if (threadIdx.x == 0 && *abort_flag && a.status) atomicOr(a.status, LIGHTKV_STATUS_TIMEOUT);
 }
@@ -249,7 +257,7 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   if (!make_map_bhnd(&qm, a->q, L.head_dim, rows, L.n_q_heads, L.batch, a->q_row_stride, a->q_head_stride,
                      a->q_batch_stride, 128) ||
       !make_map_bhnd(&km, a->k, L.head_dim, rows, L.n_kv_heads, L.batch, a->k_row_stride, a->k_head_stride,
-                     a->k_batch_stride, 128))
+                     a->k_batch_stride, XT_KEY_TILE))
     return cudaErrorInvalidValue;
   XiTcArgs x;
   x.n_vis = a->n_vis; x.xi_h = L.ws.xi_h; x.status = a->status; x.cap_in = L.ws.cap_in;
@@ -258,14 +266,15 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   x.n_q_heads = L.n_q_heads; x.group = L.n_q_heads / L.n_kv_heads;
   x.scale2 = 1.4426950408889634f / sqrtf((float)L.head_dim);
   const dim3 grid((L.ws.cap_in + 127) / 128, L.n_q_heads, L.batch);
-  const size_t smem = size_t(L.head_dim / 64) * 16384 * (1 + XT_STAGES) + 1024 + 256;
+  constexpr int BK = XT_KEY_TILE;
+  const size_t smem = size_t(L.head_dim / 64) * (16384 + size_t(XT_STAGES) * BK * 128) + 1024 + 256;
   cudaError_t e;
   if (L.head_dim == 128) {
-    if ((e = cudaFuncSetAttribute(xi_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    xi_tc_kernel<128><<<grid, 192, smem, L.stream>>>(qm, km, x);
+    if ((e = cudaFuncSetAttribute(xi_tc_kernel<128, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    xi_tc_kernel<128, BK><<<grid, 192, smem, L.stream>>>(qm, km, x);
   } else {
-    if ((e = cudaFuncSetAttribute(xi_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    xi_tc_kernel<64><<<grid, 192, smem, L.stream>>>(qm, km, x);
+    if ((e = cudaFuncSetAttribute(xi_tc_kernel<64, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    xi_tc_kernel<64, BK><<<grid, 192, smem, L.stream>>>(qm, km, x);
   }
   return cudaGetLastError();
 }
