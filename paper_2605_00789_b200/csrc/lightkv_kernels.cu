@@ -524,7 +524,7 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   const int cs = CLUSTER ? (int)tc::cluster_nctarank() : 1, rank = CLUSTER ? (int)tc::cluster_ctarank() : 0;
   auto sync_all = [&]() { if (CLUSTER) tc::cluster_sync(); else __syncthreads(); };
   const int b = blockIdx.x / cs, tid = threadIdx.x, nthr = blockDim.x;
-  const int gtid = rank * nthr + tid, gthr = cs * nthr;      // thread index / count inside the cluster
+  const int gtid = rank * nthr + tid;                        // thread index inside the cluster
   const int nW = ws.n_windows;
   int n = a.n_vis ? min(a.n_vis[b], ws.cap_in) : ws.cap_in;
   if (n < 0) n = 0;
@@ -532,8 +532,6 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   const int* a_off = ws.a_off + size_t(b) * (nW + 1);
   const int* tok_win = ws.tok_win + size_t(b) * ws.cap_in;
   const int* tok_l = ws.tok_l + size_t(b) * ws.cap_in;
-  const int* a_tok = ws.a_tok + size_t(b) * ws.cap_a;
-  const int* a_win = ws.a_win + size_t(b) * ws.cap_a;
   const unsigned long long* a_key = ws.a_key + size_t(b) * ws.cap_a;
   const int* b_tok = ws.b_tok + size_t(b) * ws.cap_b;
   float* xi = ws.xi + size_t(b) * ws.cap_in;
@@ -547,20 +545,16 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   int* grp_src = a.grp_src + size_t(b) * ws.cap_in;
   int* pos_out = a.pos_out + size_t(b) * a.cap_out;
 
-  // Exclusive scan of `value(i)` over i in [0, count) across the whole cluster: every CTA owns a
-  // contiguous range, counts it, learns the ranges before it through distributed shared memory, then
-  // scans its range.  emit(i, prefix) is called for every i; returns the grand total.
-  auto cluster_scan = [&](int count, int which, auto value, auto emit) {
-    const int chunk = (count + cs - 1) / cs, lo = min(count, rank * chunk), hi = min(count, lo + chunk);
+  // Every CTA of the cluster owns a contiguous range of the sample's tokens; a thread keeps the same tokens
+  // in every phase, so what it wrote for a token it may read back without a barrier.
+  const int chunk = (n + cs - 1) / cs, lo = min(n, rank * chunk), hi = min(n, lo + chunk);
+
+  // Exclusive scan of `value(i)` over the cluster: CTA `rank` owns [s_lo, s_hi) (at most s_chunk long, the
+  // same bound in every CTA), counts it, learns the ranges before it through distributed shared memory,
+  // then scans it.  emit(i, prefix) is called for every i; returns the grand total.
+  auto cluster_scan = [&](int s_lo, int s_hi, int s_chunk, int which, auto value, auto emit) {
     int before = 0, grand = 0;
-    if (CLUSTER) {
-      int mine = 0;
-      for (int base = lo; base < hi; base += nthr) {
-        const int i = base + tid;
-        int total;
-        block_exclusive_scan(i < hi ? value(i) : 0, warp_sums, &total);
-        mine += total;
-      }
+    auto exchange = [&](int mine) {
       if (tid == 0) cta_total[which] = mine;
       tc::cluster_sync();
       for (int j = 0; j < cs; ++j) {
@@ -568,21 +562,40 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
         if (j < rank) before += t;
         grand += t;
       }
+    };
+    if (s_chunk <= nthr) {                              // one value per thread: a single pass
+      const int i = s_lo + tid;
+      int total;
+      const int ex = block_exclusive_scan(i < s_hi ? value(i) : 0, warp_sums, &total);
+      if (CLUSTER) exchange(total); else grand = total;
+      if (i < s_hi) emit(i, before + ex);
+      return grand;
+    }
+    if (CLUSTER) {
+      int mine = 0;
+      for (int base = s_lo; base < s_hi; base += nthr) {
+        const int i = base + tid;
+        int total;
+        block_exclusive_scan(i < s_hi ? value(i) : 0, warp_sums, &total);
+        mine += total;
+      }
+      exchange(mine);
     }
     int carry = before;
-    for (int base = lo; base < hi; base += nthr) {
+    for (int base = s_lo; base < s_hi; base += nthr) {
       const int i = base + tid;
-      const int v = i < hi ? value(i) : 0;
       int total;
-      const int ex = block_exclusive_scan(v, warp_sums, &total);
-      if (i < hi) emit(i, carry + ex);
+      const int ex = block_exclusive_scan(i < s_hi ? value(i) : 0, warp_sums, &total);
+      if (i < s_hi) emit(i, carry + ex);
       carry += total;
     }
     return CLUSTER ? grand : carry;
   };
 
-  // phase 0
-  for (int i = gtid; i < n; i += gthr) {
+  // phase 1: xi of every token; every A token (even local rank, entry a_off[w] + l / 2) decides whether it is
+  // among the r lowest-FD entries of its window and, if so, takes the partner FD found for it
+  const uint32_t* key_word = reinterpret_cast<const uint32_t*>(a_key);   // [2e]: best B entry, [2e + 1]: orderable FD
+  for (int i = lo + tid; i < hi; i += nthr) {
     float v;
     if (a.xi_mode == LIGHTKV_XI_GIVEN) v = a.xi_in[size_t(b) * ws.cap_in + i];
     else if (a.xi_mode == LIGHTKV_XI_UNIFORM) v = 1.0f;
@@ -593,39 +606,43 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     }
     xi[i] = v;
     if (a.xi_out) a.xi_out[size_t(b) * ws.cap_in + i] = v;
-    partner[i] = -1;
-  }
-  sync_all();
-
-  // phase 1
-  const int n_a = a_off[nW];
-  for (int e = gtid; e < n_a; e += gthr) {
-    const int w = a_win[e];
-    const int e_lo = a_off[w], e_hi = a_off[w + 1];
-    const int r = removal_count(win_off[w + 1] - win_off[w], a.keep);
-    bool sel;
-    if (r <= 0) sel = false;
-    else if (r >= e_hi - e_lo) sel = true;
-    else {
-      // order by (lowest FD, A entry index): the high word of a_key is the orderable FD
-      const unsigned long long key = (a_key[e] & 0xffffffff00000000ull) | (unsigned)e;
-      int rk = 0;
-      for (int e2 = e_lo; e2 < e_hi; ++e2) {
-        const unsigned long long k2 = (a_key[e2] & 0xffffffff00000000ull) | (unsigned)e2;
-        rk += (k2 < key);
+    int p = -1;
+    const int l = tok_l[i];
+    if (!(l & 1)) {
+      const int w = tok_win[i];
+      const int e_lo = a_off[w], e_hi = a_off[w + 1], e = e_lo + (l >> 1);
+      if (e < ws.cap_a) {
+        const int r = removal_count(win_off[w + 1] - win_off[w], a.keep);
+        bool sel;
+        if (r <= 0) sel = false;
+        else if (r >= e_hi - e_lo) sel = true;
+        else {
+          // rank in the order (lowest FD, A entry index): entries before e win ties, entries after e lose them
+          const uint32_t mine = key_word[2 * e + 1];
+          int rk = 0;
+          for (int e2 = e_lo; e2 < e; ++e2) rk += (key_word[2 * e2 + 1] <= mine);
+          for (int e2 = e + 1; e2 < e_hi; ++e2) rk += (key_word[2 * e2 + 1] < mine);
+          sel = rk < r;
+        }
+        const uint32_t best_e = key_word[2 * e];
+        p = (sel && best_e != 0xffffffffu) ? b_tok[best_e] : -1;
+        a_partner[e] = p;                              // entry-indexed copy: phase 3 counts over it in order
       }
-      sel = rk < r;
     }
-    const unsigned best_e = (unsigned)(a_key[e] & 0xffffffffu);
-    const int p = (sel && best_e != 0xffffffffu) ? b_tok[best_e] : -1;
-    a_partner[e] = p;                                  // entry-indexed copy: the group loops below read it in order
-    if (p >= 0) partner[a_tok[e]] = p;
+    partner[i] = p;
   }
-  sync_all();
 
-  // phase 2
-  const int survivors = cluster_scan(n, 0, [&](int i) { return partner[i] < 0 ? 1 : 0; },
-                                     [&](int i, int prefix) { if (partner[i] < 0) slot[i] = prefix; });
+  // phase 2: output slot of every surviving token (its own tokens: no barrier needed before); the survivor
+  // opens its group with one member
+  const int survivors = cluster_scan(lo, hi, chunk, 0, [&](int i) { return partner[i] < 0 ? 1 : 0; },
+                                     [&](int i, int prefix) {
+                                       if (partner[i] >= 0) return;
+                                       slot[i] = prefix;
+                                       dst[i] = prefix;
+                                       if (prefix >= a.cap_out) return;
+                                       pos_out[prefix] = pos ? pos[i] : i;
+                                       grp_off[prefix] = 1;
+                                     });
   const int n_out = min(survivors, a.cap_out);
   if (gtid == 0) {
     a.n_vis_out[b] = n_out;
@@ -633,47 +650,49 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
   }
   sync_all();
 
-  // phase 3 + 4 (sizes written where the offsets will be)
-  for (int i = gtid; i < n; i += gthr) {
+  // phase 3: a merged token joins the group of its partner; its place in the group is the number of earlier
+  // entries of its window with the same partner (kept in slot[], which a merged token does not use otherwise)
+  for (int i = lo + tid; i < hi; i += nthr) {
     const int p = partner[i];
-    if (p >= 0) { dst[i] = slot[p]; continue; }
-    const int o = slot[i];
+    if (p < 0) continue;
+    const int o = slot[p];
     dst[i] = o;
-    if (o >= a.cap_out) continue;
-    pos_out[o] = pos ? pos[i] : i;
-    int sz = 1;
-    if (tok_l[i] & 1) {
-      const int w = tok_win[i];
-      for (int e = a_off[w]; e < a_off[w + 1]; ++e) sz += (a_partner[e] == i);
-    }
-    grp_off[o] = sz;
+    const int e_lo = a_off[tok_win[i]], e = e_lo + (tok_l[i] >> 1);
+    int rk = 0;
+    for (int e2 = e_lo; e2 < e; ++e2) rk += (a_partner[e2] == p);
+    slot[i] = rk;
+    if (o < a.cap_out) atomicAdd(&grp_off[o], 1);
   }
   sync_all();
-  const int members = cluster_scan(n_out, 1, [&](int o) { return grp_off[o]; },
+
+  // phase 4: group sizes -> group offsets
+  const int chunk_o = (n_out + cs - 1) / cs, lo_o = min(n_out, rank * chunk_o), hi_o = min(n_out, lo_o + chunk_o);
+  const int members = cluster_scan(lo_o, hi_o, chunk_o, 1, [&](int o) { return grp_off[o]; },
                                    [&](int o, int prefix) { grp_off[o] = prefix; });
   if (gtid == 0) grp_off[n_out] = members;
   sync_all();
 
-  // phase 5
-  for (int i = gtid; i < n; i += gthr) {
+  // phase 5: member lists, the surviving token first, then the merged ones in entry order
+  for (int i = lo + tid; i < hi; i += nthr) {
+    const int o = dst[i];
+    if (o >= a.cap_out) continue;
+    grp_src[grp_off[o] + (partner[i] < 0 ? 0 : 1 + slot[i])] = i;
+  }
+  sync_all();
+
+  // phase 6: weights xi_i / (sum of xi over the group), the sum taken in member order
+  for (int i = lo + tid; i < hi; i += nthr) {
     if (partner[i] >= 0) continue;
     const int o = slot[i];
     if (o >= a.cap_out) continue;
-    const int off = grp_off[o];
-    grp_src[off] = i;
-    int cnt = 1;
-    float den = xi[i];
-    if (tok_l[i] & 1) {
-      const int w = tok_win[i];
-      for (int e = a_off[w]; e < a_off[w + 1]; ++e) {
-        if (a_partner[e] == i) { const int t = a_tok[e]; grp_src[off + cnt++] = t; den += xi[t]; }
-      }
-    }
+    const int g0 = grp_off[o], g1 = grp_off[o + 1];
+    float den = 0.f;
+    for (int c = g0; c < g1; ++c) den += xi[grp_src[c]];
     if (den >= 1e-30f) {
-      for (int c = 0; c < cnt; ++c) { const int t = grp_src[off + c]; weight[t] = xi[t] / den; }
+      for (int c = g0; c < g1; ++c) { const int t = grp_src[c]; weight[t] = xi[t] / den; }
     } else {
       set_status(a.status, LIGHTKV_STATUS_ZERO_WEIGHT);
-      for (int c = 0; c < cnt; ++c) weight[grp_src[off + c]] = 1.0f / (float)cnt;
+      for (int c = g0; c < g1; ++c) weight[grp_src[c]] = 1.0f / (float)(g1 - g0);
     }
   }
 }
