@@ -150,6 +150,44 @@ def test_run_to_run_bit_repeatability():
         np.testing.assert_array_equal(a[key], b[key])
 
 
+# ---- seeded random geometries ---------------------------------------------------------------------
+
+def _random_workload(seed):
+    """Tiles, windows, keep ratios, head layout and sizes drawn from a seeded generator: ragged windows, several
+    tiles per sample, 600 to 4500 tokens (one to eight CTAs per sample in the selection kernel), hidden sizes
+    that are and are not multiples of 64, head sizes with and without a tensor-core path."""
+    rng = np.random.default_rng(7000 + seed)
+    n_tiles = int(rng.integers(1, 4))
+    big = seed % 3 == 0
+    tiles = tuple((int(rng.integers(18, 50 if big else 30)), int(rng.integers(18, 46 if big else 26)))
+                  for _ in range(n_tiles))
+    smallest = min(min(t) for t in tiles)
+    windows = tuple(sorted((int(rng.integers(1, min(7, smallest // 2))) for _ in range(3)), reverse=True))
+    n_kv = int(rng.choice([1, 2, 4]))
+    return S.Workload(name=f"rand{seed}", config_id=100 + seed, batch=int(rng.integers(1, 4)), tiles=tiles,
+                      n_text=int(rng.integers(1, 180)), hidden=int(rng.choice([64, 72, 192, 320, 520])),
+                      n_q_heads=n_kv * int(rng.choice([1, 2])), n_kv_heads=n_kv,
+                      head_dim=int(rng.choice([64, 128, 128, 32])), n_layers=16, layers=(3, 7, 11),
+                      windows=windows, keep=tuple(float(k) for k in rng.uniform(0.5, 0.9, size=3).round(2)))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_geometry(seed):
+    wl = _random_workload(seed)
+    H.run_schedule(wl, xi_mode=["attn", "given", "lse"][seed % 3], dtype="fp32" if seed == 4 else "bf16",
+                   engine="simt" if seed == 4 else "auto")
+
+
+def test_selection_over_eight_ctas_ragged_windows():
+    # 4480 tokens per sample (a cluster of eight CTAs in the selection kernel), windows that do not divide
+    # the grid, a single large window at the last stage (1344 tokens: the per-window rank loops at length)
+    wl = S.Workload(name="sel8", config_id=120, batch=2, tiles=((70, 64),), n_text=9, hidden=64, n_q_heads=2,
+                    n_kv_heads=1, head_dim=64, n_layers=16, layers=(3, 7, 11), windows=(6, 3, 1),
+                    keep=(0.6, 0.5, 0.7))
+    stats = H.run_schedule(wl, xi_mode="given")
+    assert stats[0]["n_out"][0] < 4480 * 0.6 + 40
+
+
 # ---- full benchmark shapes, compared on the samples the oracle can finish in seconds -----------------
 
 def test_cfg2_full_size_sampled():
