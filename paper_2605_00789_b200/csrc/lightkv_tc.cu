@@ -49,12 +49,14 @@ static bool make_map_bhnd(CUtensorMap* map, const void* base, int width, int row
 // xi per head on tensor cores (Eq. "attention-factor" over the causal softmax rows of Eq.
 // "attention-matrix").
 //
-// One CTA per (tile of 128 vision queries, head, sample); two CTAs share an SM.  Warp 0 streams the Q tile
-// once and the K tiles through a 2-stage ring with TMA; warp 1 issues S = Q K^T (128 x 128 x dh, bf16 ->
-// fp32) into one of two TMEM accumulators; warps 2-5 own one query row per thread (= TMEM lane), pull the
-// 128 logits of the row into registers, release the accumulator, and fold them into a running maximum and
-// two running sums (all visible keys / prompt keys J).  Only tiles that straddle the diagonal are masked
-// and only tiles that reach into J take the prompt-sum path.  Output per head: sum_J / sum_all.
+// A work item is (tile of 128 vision queries, head, sample); three CTAs share an SM.  Warp 0 streams the Q
+// tile once and the K tiles (64 keys) through a 2-stage ring with TMA; warp 1 issues S = Q K^T (128 x 64 x dh,
+// bf16 -> fp32) into one of two TMEM accumulators; warps 2-5 own one query row per thread (= TMEM lane), pull
+// the 64 logits of the row into registers, release the accumulator, and fold them into a running maximum and
+// two running sums (all visible keys / prompt keys J).  Tiles that straddle the diagonal are masked, and the
+// columns no row of a warp can see are skipped; only tiles that reach into J take the prompt-sum path.
+// Output per head: sum_J / sum_all.  With the caller's row log-sum-exp only the prompt key tiles are visited
+// and the CTAs walk the item list (WALK), so that an item's loads overlap the previous item's arithmetic.
 // ======================================================================================================
 __device__ __forceinline__ float ex2(float x) {          // one MUFU op, flush-to-zero
   float y;
@@ -69,13 +71,14 @@ struct XiTcArgs {
   const float* lse;                  // [B, H, N] row log-sum-exp (natural log) from the caller, or nullptr
   int64_t lse_bs, lse_hs;
   int cap_in, vis_begin, text_begin, text_end, n_q_heads, group;
+  int batch, n_qt;                   // samples, query tiles of 128 rows per (sample, head)
   float scale2;                      // log2(e) / sqrt(dh)
 };
 
 constexpr int XT_STAGES = 2;
 constexpr int XT_KEY_TILE = 64;      // keys per tile (64: three CTAs per SM; 128: two)
 
-template <int DH, int BK>
+template <int DH, int BK, bool WALK>
 __global__ void __launch_bounds__(192, BK == 64 ? 3 : 2)
 xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, XiTcArgs a) {
   constexpr int HALVES = DH / 64;
@@ -93,24 +96,43 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   uint64_t* k_empty = k_full + XT_STAGES;      // [XT_STAGES]
   uint64_t* s_full = k_empty + XT_STAGES;      // [2]
   uint64_t* s_empty = s_full + 2;              // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_empty + 2);
+  uint64_t* q_empty = s_empty + 2;             // every MMA that reads the Q tile has completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_empty + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-  const int qt = gridDim.x - 1 - blockIdx.x;   // longest rows first
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int n = a.n_vis ? min(a.n_vis[b], a.cap_in) : a.cap_in;
-  const int t0 = qt * 128;
-  if (t0 >= n) return;
-  const int nq = min(128, n - t0);
-  const int s_first = a.vis_begin + t0, s_last = s_first + nq - 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // Work items: (query tile, head, sample), the query tiles of one head next to each other (they share its K
+  // in L2), longest rows first.  WALK = false: one item per CTA, grid (query tiles, heads, samples).
+  // WALK = true: CTA c takes items c, c + gridDim.x, ... of the flattened list; every role walks the list
+  // with the same tests, so their barrier phases stay in step.
+  const int n_items = WALK ? a.n_qt * a.n_q_heads * a.batch : 0;
   // key tiles to visit: all tiles up to the last query's own key, or, when the caller supplies the row
   // log-sum-exp, only the tiles that hold prompt keys (J lies before the vision block, so it is visible)
   const int kt_lo = a.lse ? a.text_begin / BK : 0;
-  const int nkt = a.lse ? (a.text_end > a.text_begin ? (a.text_end - 1) / BK + 1 - kt_lo : 0) : s_last / BK + 1;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nkt_lse = a.text_end > a.text_begin ? (a.text_end - 1) / BK + 1 - kt_lo : 0;
+  struct Item { int h, b, t0, nq, s_first, nkt; };
+  auto decode = [&](int item, Item& it) -> bool {
+    int qt;
+    if (WALK) {
+      const int hb = item / a.n_qt;
+      qt = a.n_qt - 1 - item % a.n_qt; it.h = hb % a.n_q_heads; it.b = hb / a.n_q_heads;
+    } else {
+      qt = gridDim.x - 1 - blockIdx.x; it.h = blockIdx.y; it.b = blockIdx.z;
+    }
+    const int n = a.n_vis ? min(a.n_vis[it.b], a.cap_in) : a.cap_in;
+    it.t0 = qt * 128;
+    if (it.t0 >= n) return false;
+    it.nq = min(128, n - it.t0);
+    it.s_first = a.vis_begin + it.t0;
+    it.nkt = a.lse ? nkt_lse : (it.s_first + it.nq - 1) / BK + 1;
+    return true;
+  };
+  Item it0 = {};
+  if (!WALK && !decode(0, it0)) return;        // one item per CTA: decoded once, before the set-up
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
+    if (WALK) mbar_init(q_empty, 1);
     for (int i = 0; i < XT_STAGES; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4); }
     *abort_flag = 0;
@@ -126,118 +148,180 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     if (lane == 0) {
       prefetch_tensormap(&q_map);
       prefetch_tensormap(&k_map);
-      mbar_expect_tx(q_full, TILE_BYTES);
+      uint32_t kf = 0, done = 0;                       // K tiles fetched / items started by this CTA
+      bool ok = true;
+      for (int item = blockIdx.x; ok && (!WALK || item < n_items); item += gridDim.x) {
+        Item it = it0;
+        if ((WALK && !decode(item, it)) || it.nkt == 0) { if (WALK) continue; else break; }
+        // the Q tile is free once every MMA of the previous item has completed
+        if (WALK && done > 0 && !mbar_wait(q_empty, (done - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(q_full, TILE_BYTES);
 #pragma unroll
-      for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, s_first, h, b);
-      const int hk = h / a.group;
-      for (int kt = 0; kt < nkt; ++kt) {
-        const int s = kt % XT_STAGES;
-        if (!mbar_wait(&k_empty[s], ((kt / XT_STAGES) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(&k_full[s], KT_BYTES);
+        for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.s_first, it.h, it.b);
+        const int hk = it.h / a.group;
+        for (int kt = 0; kt < it.nkt; ++kt, ++kf) {
+          const uint32_t s = kf % XT_STAGES;
+          if (!mbar_wait(&k_empty[s], ((kf / XT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(&k_full[s], KT_BYTES);
 #pragma unroll
-        for (int hf = 0; hf < HALVES; ++hf)
-          tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, b);
+          for (int hf = 0; hf < HALVES; ++hf)
+            tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, it.b);
+        }
+        ++done;
+        if (!WALK) break;
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16(128, BK);
       const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s);
-      bool ok = mbar_wait(q_full, 0, abort_flag);
-      for (int kt = 0; ok && kt < nkt; ++kt) {
-        const int s = kt % XT_STAGES, buf = kt & 1;
-        if (!mbar_wait(&s_empty[buf], ((kt >> 1) & 1) ^ 1, abort_flag)) break;
-        if (!mbar_wait(&k_full[s], (kt / XT_STAGES) & 1, abort_flag)) break;
-        tc_fence_after();
+      uint32_t kc = 0, done = 0;                       // K tiles consumed / items started
+      bool ok = true;
+      for (int item = blockIdx.x; ok && (!WALK || item < n_items); item += gridDim.x) {
+        Item it = it0;
+        if ((WALK && !decode(item, it)) || it.nkt == 0) { if (WALK) continue; else break; }
+        if (!mbar_wait(q_full, done & 1, abort_flag)) break;
+        for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
+          const uint32_t s = kc % XT_STAGES, buf = kc & 1;
+          if (!mbar_wait(&s_empty[buf], ((kc >> 1) & 1) ^ 1, abort_flag) ||
+              !mbar_wait(&k_full[s], (kc / XT_STAGES) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk) {
-          umma_bf16(tmem_base + buf * BK, smem_desc_sw128(q_addr + (kk >> 2) * 16384 + (kk & 3) * 32),
-                    smem_desc_sw128(k_addr + s * KT_BYTES + (kk >> 2) * KHALF_BYTES + (kk & 3) * 32), idesc, kk > 0);
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            umma_bf16(tmem_base + buf * BK, smem_desc_sw128(q_addr + (kk >> 2) * 16384 + (kk & 3) * 32),
+                      smem_desc_sw128(k_addr + s * KT_BYTES + (kk >> 2) * KHALF_BYTES + (kk & 3) * 32), idesc, kk > 0);
+          }
+          umma_commit(&k_empty[s]);
+          umma_commit(&s_full[buf]);
         }
-        umma_commit(&k_empty[s]);
-        umma_commit(&s_full[buf]);
+        if (WALK && ok) umma_commit(q_empty);
+        ++done;
+        if (!WALK) break;
       }
     }
   } else {
     const int quad = warp & 3;                          // TMEM lanes this warp may read
     const int r = quad * 32 + lane;                     // query row of this thread
     const uint32_t lane_addr = tmem_base + (uint32_t(quad * 32) << 16);
-    float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
     const float sc = a.scale2;
-    for (int kt = 0; kt < nkt; ++kt) {
-      const int buf = kt & 1, j0 = (kt_lo + kt) * BK;
-      const bool landed = mbar_wait(&s_full[buf], (kt >> 1) & 1, abort_flag);
-      if (!__all_sync(0xffffffffu, landed)) break;        // the TMEM loads below are warp-wide
-      tc_fence_after();
-      float v[NC][32];
+    uint32_t kc = 0;                                    // key tiles consumed by this CTA so far
+    bool alive = true;
+    for (int item = blockIdx.x; alive && (!WALK || item < n_items); item += gridDim.x) {
+      Item it = it0;
+      if (WALK && !decode(item, it)) continue;
+      const int h = it.h, b = it.b, nq = it.nq, s_first = it.s_first;
+      float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
+      for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
+        const uint32_t buf = kc & 1;
+        const int j0 = (kt_lo + kt) * BK;
+        const bool landed = mbar_wait(&s_full[buf], (kc >> 1) & 1, abort_flag);
+        if (!__all_sync(0xffffffffu, landed)) { alive = false; break; }   // the TMEM loads below are warp-wide
+        tc_fence_after();
+        float v[NC][32];
 #pragma unroll
-      for (int c = 0; c < NC; ++c) tmem_ld32(lane_addr + buf * BK + c * 32, v[c]);
-      tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s_empty[buf]);
+        for (int c = 0; c < NC; ++c) tmem_ld32(lane_addr + buf * BK + c * 32, v[c]);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[buf]);
 
-      if (a.lse) {                                      // normaliser known: only the prompt columns count
-        const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
-        const int lo = a.text_begin - j0, hi = a.text_end - j0;
-        float st = 0.f;
+        if (a.lse) {                                      // normaliser known: only the prompt columns count
+          const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
+          const int lo = a.text_begin - j0, hi = a.text_end - j0;
+          float st = 0.f;
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
+          for (int c = 0; c < NC; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c * 32 + i >= lo && c * 32 + i < hi) st += ex2(fmaf(v[c][i], sc, -l2));
-        l_txt += st;
-        l_all = 1.f;
-        continue;
-      }
-      if (j0 + BK - 1 > s_first) {                         // tile straddles the diagonal: causal mask
-        const int lim = s_first + r - j0;               // last visible column of this row
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i >= lo && c * 32 + i < hi) st += ex2(fmaf(v[c][i], sc, -l2));
+          l_txt += st;
+          l_all = 1.f;
+          continue;
+        }
+        const bool in_j = j0 < a.text_end && j0 + BK > a.text_begin;   // tile reaches into the prompt set J
+        if (j0 + BK - 1 > s_first) {
+          // ---- tile straddles the diagonal: causal mask.  Columns beyond the warp's last visible one are skipped
+          // in blocks of eight (a warp-uniform test), so most of the masked half costs no exponentials.
+          const int lim = s_first + r - j0;               // last visible column of this row (may be negative)
+          const int lim_max = __reduce_max_sync(0xffffffffu, lim);
+          if (lim_max < 0) continue;                      // no row of this warp sees any key of the tile
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
+          for (int c = 0; c < NC; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c * 32 + i > lim) v[c][i] = -INFINITY;
-      }
-      float mxc[NC];                                     // one dependency chain per 32-column chunk
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i > lim) v[c][i] = -INFINITY;
+          if (!in_j) {
+            float mxd[NC];
 #pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        mxc[c] = v[c][0];
+            for (int c = 0; c < NC; ++c) {
+              mxd[c] = v[c][0];
 #pragma unroll
-        for (int i = 1; i < 32; ++i) mxc[c] = fmaxf(mxc[c], v[c][i]);
-      }
-      float m_new = m_run;
+              for (int i = 1; i < 32; ++i) mxd[c] = fmaxf(mxd[c], v[c][i]);
+            }
+            float m_new = m_run;                            // finite from the second tile on; tile 0 shows key 0 to every row
 #pragma unroll
-      for (int c = 0; c < NC; ++c) m_new = fmaxf(m_new, mxc[c]);
-      const float ms = m_new * sc;
-      float sa = 0.f, st = 0.f;
-      if (j0 < a.text_end && j0 + BK > a.text_begin) {   // tile reaches into the prompt set J
-        const int lo = a.text_begin - j0, hi = a.text_end - j0;
+            for (int c = 0; c < NC; ++c) m_new = fmaxf(m_new, mxd[c]);
+            const float ms = m_new * sc;
+            float sa = 0.f;
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
+            for (int c = 0; c < NC; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float p = ex2(fmaf(v[c][i], sc, -ms));
-            sa += p;
-            if (c * 32 + i >= lo && c * 32 + i < hi) st += p;
+              for (int blk = 0; blk < 4; ++blk)
+                if (c * 32 + blk * 8 <= lim_max) {
+                  float part = 0.f;
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) part += ex2(fmaf(v[c][blk * 8 + i], sc, -ms));
+                  sa += part;
+                }
+            const float resc = ex2((m_run - m_new) * sc);
+            l_all = fmaf(l_all, resc, sa);
+            l_txt *= resc;
+            m_run = m_new;
+            continue;
           }
-      } else {
-        float part[NC];                                   // independent sums
+        }
+        float mxc[NC];                                     // one dependency chain per 32-column chunk
 #pragma unroll
-        for (int c = 0; c < NC; ++c) part[c] = 0.f;
+        for (int c = 0; c < NC; ++c) {
+          mxc[c] = v[c][0];
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
+          for (int i = 1; i < 32; ++i) mxc[c] = fmaxf(mxc[c], v[c][i]);
+        }
+        float m_new = m_run;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) part[c] += ex2(fmaf(v[c][i], sc, -ms));
+        for (int c = 0; c < NC; ++c) m_new = fmaxf(m_new, mxc[c]);
+        const float ms = m_new * sc;
+        float sa = 0.f, st = 0.f;
+        if (in_j) {
+          const int lo = a.text_begin - j0, hi = a.text_end - j0;
 #pragma unroll
-        for (int c = 0; c < NC; ++c) sa += part[c];
+          for (int c = 0; c < NC; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float p = ex2(fmaf(v[c][i], sc, -ms));
+              sa += p;
+              if (c * 32 + i >= lo && c * 32 + i < hi) st += p;
+            }
+        } else {
+          float part[NC];                                   // independent sums
+#pragma unroll
+          for (int c = 0; c < NC; ++c) part[c] = 0.f;
+#pragma unroll
+          for (int c = 0; c < NC; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) part[c] += ex2(fmaf(v[c][i], sc, -ms));
+#pragma unroll
+          for (int c = 0; c < NC; ++c) sa += part[c];
+        }
+        const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
+        l_all = fmaf(l_all, resc, sa);
+        l_txt = fmaf(l_txt, resc, st);
+        m_run = m_new;
       }
-      const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
-      l_all = fmaf(l_all, resc, sa);
-      l_txt = fmaf(l_txt, resc, st);
-      m_run = m_new;
+      if (alive && r < nq && !*abort_flag)
+        a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + it.t0 + r] = a.lse ? l_txt : l_txt / l_all;
+      if (!WALK) break;
     }
-    if (r < nq && !*abort_flag)
-      a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + t0 + r] = a.lse ? l_txt : l_txt / l_all;
   }
   tc_fence_before();
   __syncthreads();
@@ -249,6 +333,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
 }
 
 bool tc_xi_supported(int head_dim) { return head_dim == 64 || head_dim == 128; }
+
+static int sm_count();
 
 cudaError_t launch_xi_tc(const LayerLaunch& L) {
   const lightkv_layer_args_t* a = L.a;
@@ -265,18 +351,26 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   x.vis_begin = a->vis_begin; x.text_begin = a->text_begin; x.text_end = a->text_end;
   x.n_q_heads = L.n_q_heads; x.group = L.n_q_heads / L.n_kv_heads;
   x.scale2 = 1.4426950408889634f / sqrtf((float)L.head_dim);
-  const dim3 grid((L.ws.cap_in + 127) / 128, L.n_q_heads, L.batch);
+  x.batch = L.batch; x.n_qt = (L.ws.cap_in + 127) / 128;
+  // One CTA per work item when the rows are long (the hardware balances them, and kernels on other streams
+  // find room as CTAs retire).  With the caller's log-sum-exp an item is two or three key tiles, all items
+  // alike: then as many CTAs as stay resident (three per SM) walk the list, and the next item's loads hide
+  // behind the current one's arithmetic.
+  const bool walk = x.lse != nullptr;
+  const long long n_items = (long long)x.n_qt * L.n_q_heads * L.batch;
+  if (n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
+  const dim3 grid = walk ? dim3((unsigned)std::min<long long>(n_items, (XT_KEY_TILE == 64 ? 3 : 2) * sm_count()))
+                         : dim3(x.n_qt, L.n_q_heads, L.batch);
   constexpr int BK = XT_KEY_TILE;
   const size_t smem = size_t(L.head_dim / 64) * (16384 + size_t(XT_STAGES) * BK * 128) + 1024 + 256;
-  cudaError_t e;
-  if (L.head_dim == 128) {
-    if ((e = cudaFuncSetAttribute(xi_tc_kernel<128, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    xi_tc_kernel<128, BK><<<grid, 192, smem, L.stream>>>(qm, km, x);
-  } else {
-    if ((e = cudaFuncSetAttribute(xi_tc_kernel<64, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    xi_tc_kernel<64, BK><<<grid, 192, smem, L.stream>>>(qm, km, x);
-  }
-  return cudaGetLastError();
+  auto launch = [&](auto kernel) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, 192, smem, L.stream>>>(qm, km, x);
+    return cudaGetLastError();
+  };
+  if (L.head_dim == 128) return walk ? launch(xi_tc_kernel<128, BK, true>) : launch(xi_tc_kernel<128, BK, false>);
+  return walk ? launch(xi_tc_kernel<64, BK, true>) : launch(xi_tc_kernel<64, BK, false>);
 }
 
 // ======================================================================================================
