@@ -829,7 +829,7 @@ constexpr int KV_THREADS = 256;
 __device__ inline int div_magic(int n, unsigned m) { return (int)__umulhi((unsigned)n, m); }
 
 template <typename T>
-__global__ void __launch_bounds__(KV_THREADS, 6)
+__global__ void __launch_bounds__(KV_THREADS, sizeof(T) == 2 ? 5 : 4)
 kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* __restrict__ k_dst,
                   T* __restrict__ v_dst, KvAddr sa, KvAddr da, int n_kv_heads, int dh, int vis_begin,
                   int n_text_after, int cap_in, int cap_out, int gather, unsigned magic_ch,
@@ -855,41 +855,69 @@ kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* _
   if (text || g1 - g0 == 1) {                                       // copy: text, lone survivor, gather mode
     const int64_t s_tok = text ? sa.token(b, row < vis_begin ? row : row - n_out + n_in)
                                : sa.token(b, vis_begin + gs[g0]);
-    for (int u = threadIdx.x; u < units; u += blockDim.x) {
-      const int kv = u >= per_kv ? 1 : 0, rem = u - kv * per_kv, h = div_magic(rem, magic_ch), c = rem - h * ch;
-      st_stream16((kv ? v_dst : k_dst) + d_tok + int64_t(h) * da.head_stride + c * V,
-                  ld_stream16((kv ? v_src : k_src) + s_tok + int64_t(h) * sa.head_stride + c * V));
+    for (int u0 = threadIdx.x; u0 < units; u0 += 4 * blockDim.x) {   // four units' loads in flight per thread
+      uint4 v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int u = u0 + q * blockDim.x;
+        if (u < units) {
+          const int kv = u >= per_kv ? 1 : 0, rem = u - kv * per_kv, h = div_magic(rem, magic_ch), c = rem - h * ch;
+          v[q] = ld_stream16((kv ? v_src : k_src) + s_tok + int64_t(h) * sa.head_stride + c * V);
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int u = u0 + q * blockDim.x;
+        if (u < units) {
+          const int kv = u >= per_kv ? 1 : 0, rem = u - kv * per_kv, h = div_magic(rem, magic_ch), c = rem - h * ch;
+          st_stream16((kv ? v_dst : k_dst) + d_tok + int64_t(h) * da.head_stride + c * V, v[q]);
+        }
+      }
     }
     return;
   }
-  for (int u = threadIdx.x; u < units; u += blockDim.x) {
-    const int kv = u >= per_kv ? 1 : 0, rem = u - kv * per_kv, h = div_magic(rem, magic_ch), c = rem - h * ch;
-    const T* sp = (kv ? v_src : k_src) + int64_t(h) * sa.head_stride + c * V;
-    float acc[V];
+  // merge: two units per thread and two members at a time, i.e. four loads in flight whatever the group's size
+  for (int u0 = threadIdx.x; u0 < units; u0 += 2 * blockDim.x) {
+    const int u1 = u0 + blockDim.x;
+    const bool two = u1 < units;
+    const int kv0 = u0 >= per_kv ? 1 : 0, rem0 = u0 - kv0 * per_kv, h0 = div_magic(rem0, magic_ch), c0 = rem0 - h0 * ch;
+    const int ub = two ? u1 : u0;
+    const int kv1 = ub >= per_kv ? 1 : 0, rem1 = ub - kv1 * per_kv, h1 = div_magic(rem1, magic_ch), c1 = rem1 - h1 * ch;
+    const T* sp0 = (kv0 ? v_src : k_src) + int64_t(h0) * sa.head_stride + c0 * V;
+    const T* sp1 = (kv1 ? v_src : k_src) + int64_t(h1) * sa.head_stride + c1 * V;
+    float acc0[V], acc1[V];
 #pragma unroll
-    for (int j = 0; j < V; ++j) acc[j] = 0.f;
-    for (int g = g0; g < g1; g += 4) {                              // up to four members' loads in flight
-      uint4 v[4];
-      float wv[4];
+    for (int j = 0; j < V; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
+    for (int g = g0; g < g1; g += 2) {
+      uint4 va[2], vb[2];
+      float wv[2];
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
+      for (int m = 0; m < 2; ++m) {
         if (g + m < g1) {
           const int i = gs[g + m];
           wv[m] = wt[i];
-          v[m] = ld_stream16(sp + sa.token(b, vis_begin + i));
+          const int64_t tok = sa.token(b, vis_begin + i);
+          va[m] = ld_stream16(sp0 + tok);
+          if (two) vb[m] = ld_stream16(sp1 + tok);
         }
       }
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
+      for (int m = 0; m < 2; ++m) {
         if (g + m < g1) {
           float f[V];
-          unpack16(v[m], f, T());
+          unpack16(va[m], f, T());
 #pragma unroll
-          for (int j = 0; j < V; ++j) acc[j] = fmaf(wv[m], f[j], acc[j]);
+          for (int j = 0; j < V; ++j) acc0[j] = fmaf(wv[m], f[j], acc0[j]);
+          if (two) {
+            unpack16(vb[m], f, T());
+#pragma unroll
+            for (int j = 0; j < V; ++j) acc1[j] = fmaf(wv[m], f[j], acc1[j]);
+          }
         }
       }
     }
-    st_stream16((kv ? v_dst : k_dst) + d_tok + int64_t(h) * da.head_stride + c * V, pack16(acc, T()));
+    st_stream16((kv0 ? v_dst : k_dst) + d_tok + int64_t(h0) * da.head_stride + c0 * V, pack16(acc0, T()));
+    if (two) st_stream16((kv1 ? v_dst : k_dst) + d_tok + int64_t(h1) * da.head_stride + c1 * V, pack16(acc1, T()));
   }
 }
 
@@ -904,7 +932,8 @@ cudaError_t launch_kv_compact(const KvLaunch& K) {
   const unsigned magic_ch = (unsigned)(((1ull << 32) + ch_host - 1) / ch_host);
   const dim3 grid(a->vis_begin + K.cap_out + a->n_text_after, K.batch);
   const int units = 2 * K.n_kv_heads * ch_host;
-  const int threads = std::min(KV_THREADS, (units + 31) / 32 * 32);     // narrow caches (GQA) get narrow CTAs
+  // two units per thread (both in flight); narrow caches (GQA) get narrow CTAs
+  const int threads = std::min(KV_THREADS, ((units + 1) / 2 + 31) / 32 * 32);
   const int gather = a->mode == LIGHTKV_KV_GATHER;
   if (K.dtype == LIGHTKV_BF16)
     kv_compact_kernel<__nv_bfloat16><<<grid, threads, 0, K.stream>>>(
