@@ -747,7 +747,15 @@ merge_rows_kernel(const T* __restrict__ src, int64_t src_bs, int64_t src_rs,
   const int chunks = d / V;
   if (row < vis_begin || row >= vis_begin + n_out) {
     const T* srow = sb + size_t(row < vis_begin ? row : row - n_out + n_in) * src_rs;
-    for (int c = threadIdx.x; c < chunks; c += blockDim.x) st_stream16(orow + c * V, ld_stream16(srow + c * V));
+    for (int c0 = threadIdx.x; c0 < chunks; c0 += 2 * blockDim.x) {
+      const int c1 = c0 + blockDim.x;
+      const uint4 a0 = ld_stream16(srow + c0 * V);
+      if (c1 < chunks) {
+        const uint4 a1 = ld_stream16(srow + c1 * V);
+        st_stream16(orow + c1 * V, a1);
+      }
+      st_stream16(orow + c0 * V, a0);
+    }
     return;
   }
   const int o = row - vis_begin;
@@ -756,32 +764,43 @@ merge_rows_kernel(const T* __restrict__ src, int64_t src_bs, int64_t src_rs,
   const int* gs = grp_src + size_t(b) * cap_in;
   const float* wt = weight + size_t(b) * cap_in;
   const T* vis = sb + size_t(vis_begin) * src_rs;
-  for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
-    float acc[V];
+  // two 16-byte chunks per thread and two members at a time: four loads in flight whatever the group's size
+  for (int c0 = threadIdx.x; c0 < chunks; c0 += 2 * blockDim.x) {
+    const int c1 = c0 + blockDim.x;
+    const bool two = c1 < chunks;
+    float acc0[V], acc1[V];
 #pragma unroll
-    for (int j = 0; j < V; ++j) acc[j] = 0.f;
-    for (int g = g0; g < g1; g += 4) {
-      uint4 v[4];
-      float wv[4];
+    for (int j = 0; j < V; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
+    for (int g = g0; g < g1; g += 2) {
+      uint4 va[2], vb[2];
+      float wv[2];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 2; ++u) {
         if (g + u < g1) {
           const int i = gs[g + u];
           wv[u] = wt[i];
-          v[u] = ld_stream16(vis + size_t(i) * src_rs + c * V);
+          const T* r = vis + size_t(i) * src_rs;
+          va[u] = ld_stream16(r + c0 * V);
+          if (two) vb[u] = ld_stream16(r + c1 * V);
         }
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 2; ++u) {
         if (g + u < g1) {
           float f[V];
-          unpack16(v[u], f, T());
+          unpack16(va[u], f, T());
 #pragma unroll
-          for (int j = 0; j < V; ++j) acc[j] = fmaf(wv[u], f[j], acc[j]);
+          for (int j = 0; j < V; ++j) acc0[j] = fmaf(wv[u], f[j], acc0[j]);
+          if (two) {
+            unpack16(vb[u], f, T());
+#pragma unroll
+            for (int j = 0; j < V; ++j) acc1[j] = fmaf(wv[u], f[j], acc1[j]);
+          }
         }
       }
     }
-    st_stream16(orow + c * V, pack16(acc, T()));
+    st_stream16(orow + c0 * V, pack16(acc0, T()));
+    if (two) st_stream16(orow + c1 * V, pack16(acc1, T()));
   }
 }
 
