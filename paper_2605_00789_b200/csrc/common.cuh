@@ -133,4 +133,14 @@ __device__ inline uint32_t orderable(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Programmatic dependent launch.  Every kernel of the library is launched with programmatic stream
+// serialization and begins with this call: it lets the next kernel of the stream become resident, then
+// waits until the kernel before this one has completed and its writes are visible.  So a kernel's launch
+// latency hides behind its predecessor, and nothing is read or written before the predecessor is done.
+// Launched without the attribute, both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 }  // namespace lkv

@@ -22,6 +22,7 @@ __device__ inline void set_status(uint32_t* status, uint32_t bit) {
 __global__ void __launch_bounds__(1024)
 window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __restrict__ n_vis,
                     Workspace ws, uint32_t* status) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int nW = g.n_windows;
   uint16_t* cnt = reinterpret_cast<uint16_t*>(smem_raw);                        // [32][nW]
@@ -168,8 +169,7 @@ cudaError_t launch_window_build(const LayerLaunch& L) {
   cudaError_t e = cudaFuncSetAttribute(window_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        200 * 1024);
   if (e != cudaSuccess) return e;
-  window_build_kernel<<<L.batch, 1024, smem, L.stream>>>(L.geo, L.a->pos, L.a->n_vis, L.ws, L.a->status);
-  return cudaGetLastError();
+  return launch_kernel(window_build_kernel, L.batch, 1024, smem, L.stream, 1, L.geo, L.a->pos, L.a->n_vis, L.ws, L.a->status);
 }
 
 // =====================================================================================================
@@ -199,6 +199,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_stride, int vis_begin,
                int d, Workspace ws) {
+  grid_dependency_sync();
   __shared__ float As[FD_TA][FD_KC + 1];
   __shared__ float Bs[FD_TB][FD_KC + 1];
   __shared__ float Gs[FD_TA][FD_TB + 1];
@@ -303,14 +304,11 @@ fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_s
 cudaError_t launch_fd_simt(const LayerLaunch& L) {
   const dim3 grid((L.ws.cap_a + FD_TA - 1) / FD_TA, L.batch);
   if (L.dtype == LIGHTKV_BF16)
-    fd_simt_kernel<__nv_bfloat16><<<grid, 256, 0, L.stream>>>(
-        static_cast<const __nv_bfloat16*>(L.a->hidden), L.a->hidden_batch_stride, L.a->hidden_row_stride,
-        L.a->vis_begin, L.hidden, L.ws);
-  else
-    fd_simt_kernel<float><<<grid, 256, 0, L.stream>>>(
-        static_cast<const float*>(L.a->hidden), L.a->hidden_batch_stride, L.a->hidden_row_stride,
-        L.a->vis_begin, L.hidden, L.ws);
-  return cudaGetLastError();
+    return launch_kernel(fd_simt_kernel<__nv_bfloat16>, grid, 256, 0, L.stream, 1,
+                         static_cast<const __nv_bfloat16*>(L.a->hidden), L.a->hidden_batch_stride,
+                         L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.ws);
+  return launch_kernel(fd_simt_kernel<float>, grid, 256, 0, L.stream, 1, static_cast<const float*>(L.a->hidden),
+                       L.a->hidden_batch_stride, L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.ws);
 }
 
 // =====================================================================================================
@@ -329,6 +327,7 @@ xi_simt_kernel(const T* __restrict__ q, int64_t q_bs, int64_t q_hs, int64_t q_rs
                const float* __restrict__ lse, int64_t lse_bs, int64_t lse_hs,
                const int* __restrict__ n_vis, int vis_begin, int text_begin, int text_end,
                int n_q_heads, int n_kv_heads, int dh, Workspace ws) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int ld = dh + 1;
   float* Qs = reinterpret_cast<float*>(smem_raw);       // [XI_TQ][ld]
@@ -445,7 +444,7 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
     auto kern = xi_simt_kernel<__nv_bfloat16>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024)) != cudaSuccess)
       return e;
-    kern<<<grid, 256, smem, L.stream>>>(
+    return launch_kernel(kern, grid, 256, smem, L.stream, 1,
         static_cast<const __nv_bfloat16*>(a->q), a->q_batch_stride, a->q_head_stride, a->q_row_stride,
         static_cast<const __nv_bfloat16*>(a->k), a->k_batch_stride, a->k_head_stride, a->k_row_stride,
         lse, a->lse_batch_stride, a->lse_head_stride, a->n_vis, a->vis_begin, a->text_begin, a->text_end,
@@ -454,7 +453,7 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
     auto kern = xi_simt_kernel<float>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024)) != cudaSuccess)
       return e;
-    kern<<<grid, 256, smem, L.stream>>>(
+    return launch_kernel(kern, grid, 256, smem, L.stream, 1,
         static_cast<const float*>(a->q), a->q_batch_stride, a->q_head_stride, a->q_row_stride,
         static_cast<const float*>(a->k), a->k_batch_stride, a->k_head_stride, a->k_row_stride,
         lse, a->lse_batch_stride, a->lse_head_stride, a->n_vis, a->vis_begin, a->text_begin, a->text_end,
@@ -519,6 +518,7 @@ __device__ inline int block_exclusive_scan(int v, int* warp_sums /* [33] smem */
 // CLUSTER = false: one CTA per sample, plain launch, block barriers only.
 template <bool CLUSTER>
 __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectArgs a) {
+  grid_dependency_sync();
   __shared__ int warp_sums[33];
   __shared__ int cta_total[2];                  // survivors / group members counted by this CTA
   const int cs = CLUSTER ? (int)tc::cluster_nctarank() : 1, rank = CLUSTER ? (int)tc::cluster_ctarank() : 0;
@@ -706,21 +706,8 @@ cudaError_t launch_select_map(const LayerLaunch& L) {
   s.xi_out = a->xi_out; s.status = a->status;
   // one cluster per sample: 1, 2, 4 or 8 CTAs of 1024 threads, about one token per thread
   const int cs = L.ws.cap_in <= 1024 ? 1 : (L.ws.cap_in <= 2048 ? 2 : (L.ws.cap_in <= 4096 ? 4 : 8));
-  if (cs == 1) {
-    select_map_kernel<false><<<L.batch, 1024, 0, L.stream>>>(L.ws, s);
-    return cudaGetLastError();
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(L.batch * cs);
-  cfg.blockDim = dim3(1024);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = L.stream;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = cs; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_map_kernel<true>, L.ws, s);
+  if (cs == 1) return launch_kernel(select_map_kernel<false>, L.batch, 1024, 0, L.stream, 1, L.ws, s);
+  return launch_kernel(select_map_kernel<true>, L.batch * cs, 1024, 0, L.stream, cs, L.ws, s);
 }
 
 // =====================================================================================================
@@ -737,6 +724,7 @@ merge_rows_kernel(const T* __restrict__ src, int64_t src_bs, int64_t src_rs,
                   const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
                   const int* __restrict__ grp_off, const int* __restrict__ grp_src,
                   const float* __restrict__ weight) {
+  grid_dependency_sync();
   constexpr int V = Vec<T>::n;
   const int b = blockIdx.y, row = blockIdx.x;
   const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
@@ -809,18 +797,16 @@ cudaError_t launch_merge_rows(const LayerLaunch& L) {
   const int rows = a->vis_begin + L.ws.cap_out + a->n_text_after;
   const dim3 grid(rows, L.batch);
   if (L.dtype == LIGHTKV_BF16)
-    merge_rows_kernel<__nv_bfloat16><<<grid, 256, 0, L.stream>>>(
+    return launch_kernel(merge_rows_kernel<__nv_bfloat16>, grid, 256, 0, L.stream, 1,
         static_cast<const __nv_bfloat16*>(a->hidden), a->hidden_batch_stride, a->hidden_row_stride,
         static_cast<__nv_bfloat16*>(a->hidden_out), a->hidden_out_batch_stride, a->hidden_out_row_stride,
         L.hidden, a->vis_begin, a->n_text_after, L.ws.cap_in, L.ws.cap_out, a->n_vis, a->n_vis_out,
         a->grp_off, a->grp_src, a->weight);
-  else
-    merge_rows_kernel<float><<<grid, 256, 0, L.stream>>>(
+  return launch_kernel(merge_rows_kernel<float>, grid, 256, 0, L.stream, 1,
         static_cast<const float*>(a->hidden), a->hidden_batch_stride, a->hidden_row_stride,
         static_cast<float*>(a->hidden_out), a->hidden_out_batch_stride, a->hidden_out_row_stride,
         L.hidden, a->vis_begin, a->n_text_after, L.ws.cap_in, L.ws.cap_out, a->n_vis, a->n_vis_out,
         a->grp_off, a->grp_src, a->weight);
-  return cudaGetLastError();
 }
 
 // =====================================================================================================
@@ -855,6 +841,7 @@ kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* _
                   const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
                   const int* __restrict__ grp_off, const int* __restrict__ grp_src,
                   const float* __restrict__ weight) {
+  grid_dependency_sync();
   constexpr int V = Vec<T>::n;
   const int b = blockIdx.y, row = blockIdx.x;
   const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
@@ -955,18 +942,16 @@ cudaError_t launch_kv_compact(const KvLaunch& K) {
   const int threads = std::min(KV_THREADS, ((units + 1) / 2 + 31) / 32 * 32);
   const int gather = a->mode == LIGHTKV_KV_GATHER;
   if (K.dtype == LIGHTKV_BF16)
-    kv_compact_kernel<__nv_bfloat16><<<grid, threads, 0, K.stream>>>(
+    return launch_kernel(kv_compact_kernel<__nv_bfloat16>, grid, threads, 0, K.stream, 1,
         static_cast<const __nv_bfloat16*>(a->k_src), static_cast<const __nv_bfloat16*>(a->v_src),
         static_cast<__nv_bfloat16*>(a->k_dst), static_cast<__nv_bfloat16*>(a->v_dst), sa, da, K.n_kv_heads,
         K.head_dim, a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, magic_ch, a->n_vis,
         a->n_vis_out, a->grp_off, a->grp_src, a->weight);
-  else
-    kv_compact_kernel<float><<<grid, threads, 0, K.stream>>>(
+  return launch_kernel(kv_compact_kernel<float>, grid, threads, 0, K.stream, 1,
         static_cast<const float*>(a->k_src), static_cast<const float*>(a->v_src),
         static_cast<float*>(a->k_dst), static_cast<float*>(a->v_dst), sa, da, K.n_kv_heads, K.head_dim,
         a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, magic_ch, a->n_vis, a->n_vis_out,
         a->grp_off, a->grp_src, a->weight);
-  return cudaGetLastError();
 }
 
 }  // namespace lkv

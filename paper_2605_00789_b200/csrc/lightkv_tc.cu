@@ -81,6 +81,7 @@ constexpr int XT_KEY_TILE = 64;      // keys per tile (64: three CTAs per SM; 12
 template <int DH, int BK, bool WALK>
 __global__ void __launch_bounds__(192, BK == 64 ? 3 : 2)
 xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, XiTcArgs a) {
+  grid_dependency_sync();
   constexpr int HALVES = DH / 64;
   constexpr uint32_t TILE_BYTES = HALVES * 16384;          // Q tile: 128 rows x DH bf16
   constexpr uint32_t KHALF_BYTES = BK * 128;               // BK key rows x 64 columns
@@ -366,8 +367,7 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   auto launch = [&](auto kernel) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, 192, smem, L.stream>>>(qm, km, x);
-    return cudaGetLastError();
+    return launch_kernel(kernel, grid, 192, smem, L.stream, 1, qm, km, x);
   };
   if (L.head_dim == 128) return walk ? launch(xi_tc_kernel<128, BK, true>) : launch(xi_tc_kernel<128, BK, false>);
   return walk ? launch(xi_tc_kernel<64, BK, true>) : launch(xi_tc_kernel<64, BK, false>);
@@ -491,6 +491,9 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // barriers and tensor memory are set up while the kernel before this one may still be running; from here on
+  // global memory is read (and written), so that kernel must have completed
+  grid_dependency_sync();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t ring = smem_u32(base);
   const int nW = a.ws.n_windows;
@@ -794,22 +797,11 @@ cudaError_t launch_fd_tc(const LayerLaunch& L) {
   if (ks == 1) {
     if ((e = cudaFuncSetAttribute(fd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM)) != cudaSuccess)
       return e;
-    fd_tc_kernel<false><<<clusters, FT_LOADERS + 32, FT_SMEM, L.stream>>>(f);
-    return cudaGetLastError();
+    return launch_kernel(fd_tc_kernel<false>, clusters, FT_LOADERS + 32, FT_SMEM, L.stream, 1, f);
   }
   if ((e = cudaFuncSetAttribute(fd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM)) != cudaSuccess)
     return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(clusters * ks);
-  cfg.blockDim = dim3(FT_LOADERS + 32);
-  cfg.dynamicSmemBytes = FT_SMEM;
-  cfg.stream = L.stream;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = ks; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, fd_tc_kernel<true>, f);
+  return launch_kernel(fd_tc_kernel<true>, clusters * ks, FT_LOADERS + 32, FT_SMEM, L.stream, ks, f);
 }
 
 }  // namespace lkv
