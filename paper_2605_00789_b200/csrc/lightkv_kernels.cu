@@ -463,15 +463,20 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
 }
 
 // =====================================================================================================
-// Selection + merge map (Steps 2-5).  One cluster of 1-8 CTAs per sample (about a token per thread), phases
-// separated by cluster barriers, prefix sums across the cluster through distributed shared memory.
-//   0  xi = fixed-order sum over heads (or given / uniform)
-//   1  per window: r = removal_count(n_w); the r A entries with the smallest (FD, index) are selected
-//      (rank by counting; skipped when r = |A|); a selected A token records its best B token
-//   2  survivors (all B, unselected A) get consecutive output slots in storage (= position) order
-//   3  dst, pos_out
-//   4  group sizes -> grp_off (scan) ; 5 grp_src (survivor first, then its A members ascending) and
-//      weights xi_i / sum (summed in that fixed order)
+// Selection + merge map (Steps 2-5).  One cluster of 1-8 CTAs per sample (about a token per thread); every
+// CTA keeps a contiguous range of the sample's tokens through all phases, phases that read what other
+// threads wrote are separated by cluster barriers, prefix sums cross the cluster through distributed shared
+// memory.
+//   1  xi = fixed-order sum over heads (or given / uniform); every A token (even local rank): r =
+//      removal_count(n_w), selected iff it is among the r entries of its window with the smallest
+//      (FD, index) (rank by counting 32-bit keys; skipped when r = |A|); a selected token takes its best B
+//   2  survivors (all B, unselected A) get consecutive output slots in storage (= position) order: dst,
+//      pos_out, and a group of one member each
+//   3  a merged token joins its partner's group (integer atomic on the size); its place in the group is
+//      the number of earlier entries of its window with the same partner
+//   4  group sizes -> grp_off (scan)
+//   5  grp_src: the survivor first, then its merged A tokens in entry order
+//   6  weights xi_i / sum over the group, the sum taken in that fixed order
 // =====================================================================================================
 struct SelectArgs {
   int n_q_heads, xi_mode, cap_out;
