@@ -118,7 +118,8 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
             # scatter the contiguous K/V into shuffled pages, compact page pool -> page pool, gather back
             nblk_s = (n_seq + paged - 1) // paged
             nblk_d = (n_seq_out + paged - 1) // paged
-            mb = max(nblk_s, nblk_d)
+            # the block tables must cover the stage's capacity (the host cannot know the device-side counts)
+            mb = max(nblk_s, nblk_d, (vb + info.cap_in + n_text_after + paged - 1) // paged)
             g = torch.Generator().manual_seed(1234 + stage)
             perm_s = torch.randperm(bsz * mb, generator=g).reshape(bsz, mb).to(torch.int32)
             perm_d = torch.randperm(bsz * mb, generator=g).reshape(bsz, mb).to(torch.int32)

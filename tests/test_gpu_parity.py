@@ -174,8 +174,10 @@ def _random_workload(seed):
 @pytest.mark.parametrize("seed", range(16))
 def test_random_geometry(seed):
     wl = _random_workload(seed)
+    # K/V side: merge or gather, contiguous or paged caches (pages of 16 or 5 tokens), both cache layouts
     H.run_schedule(wl, xi_mode=["attn", "given", "lse"][seed % 3], dtype="fp32" if seed == 4 else "bf16",
-                   engine="simt" if seed == 4 else "auto")
+                   engine="simt" if seed == 4 else "auto", kv_mode=["merge", "gather"][(seed // 2) % 2],
+                   paged=[0, 16, 0, 5][seed % 4], kv_layout="bnhd" if seed % 4 == 2 else "bhnd")
 
 
 def test_selection_over_eight_ctas_ragged_windows():
