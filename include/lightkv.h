@@ -230,7 +230,8 @@ typedef struct {
   int64_t src_batch_stride, src_head_stride, src_row_stride;
   int64_t dst_batch_stride, dst_head_stride, dst_row_stride;
   int32_t page_size;               /* 0 = contiguous */
-  int32_t max_blocks;              /* row stride of the block tables */
+  int32_t max_blocks;              /* row stride of the block tables; max_blocks * page_size must cover
+                                      vis_begin + cap_in + n_text_after tokens, else INVALID_ARG */
   const int32_t* src_block_table;  /* DEVICE [B, max_blocks] */
   const int32_t* dst_block_table;  /* DEVICE [B, max_blocks] */
   int64_t src_page_stride, dst_page_stride;
