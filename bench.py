@@ -198,16 +198,21 @@ def build_inputs(wl, plan, L, torch, device, sample_offset, kv_layout="bhnd", xi
 
 def run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None, side=None, aux=None):
     """lightkv_compress_layer on the current stream, then lightkv_compact_kv either on the same stream or,
-    when `side` is given, on that stream behind an event (the compaction only needs the stage's merge map)."""
+    when `side` is given, on that stream behind the call's map event (the compaction only needs the stage's
+    merge map, which is complete before the hidden-state merge starts)."""
     import torch
     d = stg["dev"]
+    map_event = stg.get("map_event") if side is not None else None
     L.compress_layer(plan, st, d["hidden"], stg["out"], vis_begin=wl.n_text, q=d["q"], k=d["k"], n_vis=n_vis,
-                     pos=pos, trace_events=trace, aux_stream=aux, lse=d.get("lse"))
+                     pos=pos, trace_events=trace, aux_stream=aux, lse=d.get("lse"), map_event=map_event)
     if side is None:
         L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
                      n_vis=n_vis)
     else:
-        side.wait_stream(torch.cuda.current_stream())
+        if map_event is not None:
+            side.wait_event(map_event)
+        else:
+            side.wait_stream(torch.cuda.current_stream())
         L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
                      n_vis=n_vis, stream=side)
 
@@ -381,6 +386,10 @@ def main():
 
     side = torch.cuda.Stream(device=device) if args.streams == 2 else None
     aux = torch.cuda.Stream(device=device) if args.streams == 2 else None
+    if side is not None:
+        for s in stages:              # recorded by the library after the merge map of the stage is complete
+            s["map_event"] = torch.cuda.Event()
+            s["map_event"].record()   # torch creates the CUDA event lazily; the C ABI needs a live handle
     for _ in range(args.warmup):
         run_step(L, plan, wl, stages, side=side, aux=aux)
 
@@ -573,7 +582,7 @@ def main():
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
                 "us_per_compression_layer": 1e3 * ms_step / n_stages,
                 "schedule": ("streams: window build + FD beside xi inside lightkv_compress_layer (aux_stream); "
-                             "lightkv_compact_kv of stage i beside lightkv_compress_layer of stage i+1"
+                             "lightkv_compact_kv of stage i behind the stage's map event, beside its hidden-state merge and lightkv_compress_layer of stage i+1"
                              if side is not None else "one stream"),
                 "cuda_graph": step_graph is not None,
                 "ms_per_step_one_stream": ms_step_one_stream,

@@ -179,6 +179,11 @@ typedef struct {
                                       xi contraction runs on `stream`; the two are forked and joined with
                                       events inside the call, so the caller sees everything ordered on
                                       `stream` as before.  The stream must belong to the same device. */
+  void*   map_event;               /* cudaEvent_t created by the caller, or NULL.  Recorded on `stream` once
+                                      the merge map (n_vis_out, pos_out, dst, weight, grp_off, grp_src) is
+                                      complete, i.e. before the hidden-state merge: lightkv_compact_kv only
+                                      needs the map, so a caller may start it on another stream behind this
+                                      event, beside the hidden-state merge. */
 } lightkv_layer_args_t;
 
 #define LIGHTKV_TRACE_EVENTS 6

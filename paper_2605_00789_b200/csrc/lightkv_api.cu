@@ -311,6 +311,8 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
       return LIGHTKV_ERR_CUDA;
   }
   if (launch_select_map(L) != cudaSuccess || mark(4) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+  if (a->map_event && cudaEventRecord(static_cast<cudaEvent_t>(a->map_event), L.stream) != cudaSuccess)
+    return LIGHTKV_ERR_CUDA;
   if (launch_merge_rows(L) != cudaSuccess || mark(5) != cudaSuccess) return LIGHTKV_ERR_CUDA;
   return LIGHTKV_OK;
 }

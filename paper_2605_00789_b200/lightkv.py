@@ -59,7 +59,8 @@ class _LayerArgs(C.Structure):
                 ("weight", C.c_void_p), ("grp_off", C.c_void_p), ("grp_src", C.c_void_p),
                 ("xi_out", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p),
-                ("trace_events", C.POINTER(C.c_void_p)), ("seq_rows", C.c_int32), ("aux_stream", C.c_void_p)]
+                ("trace_events", C.POINTER(C.c_void_p)), ("seq_rows", C.c_int32), ("aux_stream", C.c_void_p),
+                ("map_event", C.c_void_p)]
 
 
 TRACE_EVENTS = 6
@@ -216,7 +217,7 @@ def _stream_handle(stream) -> int:
 def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin: int,
                 n_text_after: int = 0, text_begin: int = 0, text_end: Optional[int] = None,
                 q=None, k=None, lse=None, xi=None, n_vis=None, pos=None, stream=None,
-                trace_events=None, aux_stream=None) -> _LayerArgs:
+                trace_events=None, aux_stream=None, map_event=None) -> _LayerArgs:
     a = _LayerArgs()
     a.struct_size = C.sizeof(_LayerArgs)
     a.stage, a.vis_begin, a.n_text_after = stage, vis_begin, n_text_after
@@ -238,6 +239,8 @@ def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin:
     a.stream = _stream_handle(stream)
     if aux_stream is not None:
         a.aux_stream = aux_stream.cuda_stream
+    if map_event is not None:         # a torch.cuda.Event that has been recorded once (torch creates it lazily)
+        a.map_event = map_event.cuda_event
     if trace_events is not None:      # TRACE_EVENTS torch.cuda.Event objects (enable_timing=True), already created
         assert len(trace_events) == TRACE_EVENTS
         a.trace_events = (C.c_void_p * TRACE_EVENTS)(*[e.cuda_event for e in trace_events])
@@ -247,7 +250,7 @@ def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin:
 def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, **kw) -> None:
     """lightkv_compress_layer.  hidden [B,N,d]; keywords: vis_begin, n_text_after, text_begin, text_end,
     q [B,H,N,dh], k [B,H_kv,N,dh] (any strides with a contiguous last dimension), lse [B,H,N] fp32,
-    xi [B,cap_in] fp32, n_vis [B] int32, pos [B,cap_in] int32, stream, trace_events, aux_stream."""
+    xi [B,cap_in] fp32, n_vis [B] int32, pos [B,cap_in] int32, stream, trace_events, aux_stream, map_event."""
     a = _layer_args(plan, stage, hidden, out, **kw)
     _check(library().lightkv_compress_layer(plan.handle, C.byref(a)), "lightkv_compress_layer")
 

@@ -78,7 +78,7 @@ def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_t
 
 def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0, text_range=None,
               lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None, aux_stream=None,
-              kv_layout="bhnd"):
+              kv_layout="bhnd", kv_stream=None):
     """Run lightkv_compress_layer (or `layer_fn`, a binding function with the same signature) +
     lightkv_compact_kv on the device; returns numpy outputs."""
     import torch
@@ -92,6 +92,12 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
     kw = {}
     if aux_stream is not None:
         kw["aux_stream"] = aux_stream
+    kv_kw = {}
+    if kv_stream is not None:
+        # K/V compaction on a second stream behind the call's map event (recorded before the hidden-state merge)
+        kw["map_event"] = torch.cuda.Event()
+        kw["map_event"].record()
+        kv_kw["stream"] = kv_stream
     if xi_mode in ("attn", "lse"):
         kw["q"], kw["k"] = to_device(inp["q"], dtype, device), to_device(inp["k"], dtype, device)
     if xi_mode == "lse":
@@ -114,6 +120,9 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
         k_src, v_src = to_device(inp["k"], dtype, device), to_device(inp["v"], dtype, device)
         hkv, dh = k_src.shape[1], k_src.shape[3]
         mode = L.KV_MERGE if kv_mode == "merge" else L.KV_GATHER
+        if kv_stream is not None:
+            kv_stream.wait_stream(torch.cuda.current_stream())     # the K/V source tensors were just written
+            kv_stream.wait_event(kw["map_event"])
         if paged:
             # scatter the contiguous K/V into shuffled pages, compact page pool -> page pool, gather back
             nblk_s = (n_seq + paged - 1) // paged
@@ -149,7 +158,7 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
                 k_src, v_src, k_dst, v_dst = as_bnhd(k_src), as_bnhd(v_src), as_bnhd(k_dst), as_bnhd(v_dst)
                 assert k_src.stride(1) == dh and k_src.stride(2) == hkv * dh
             L.compact_kv(plan, stage, out, k_src, v_src, k_dst, v_dst, vis_begin=vb, n_text_after=n_text_after,
-                         mode=mode, n_vis=torch.from_numpy(inp["n_vis"]).to(device))
+                         mode=mode, n_vis=torch.from_numpy(inp["n_vis"]).to(device), **kv_kw)
         torch.cuda.synchronize()
         res["k_out"], res["v_out"] = k_dst.float().cpu().numpy(), v_dst.float().cpu().numpy()
     torch.cuda.synchronize()
@@ -219,7 +228,7 @@ def compare_stage(wl, stage, inp, ref, gpu, dtype="bf16", kv_mode="merge", n_tex
 
 
 def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge", paged=0, samples=None,
-                 stages=None, oracle_samples=None, aux_stream=None, kv_layout="bhnd"):
+                 stages=None, oracle_samples=None, aux_stream=None, kv_layout="bhnd", kv_stream=None):
     """All stages of a workload, chained through the surviving positions; returns per-stage stats."""
     bsz = wl.batch if samples is None else len(samples)
     plan = make_plan(wl, dtype, xi_mode, engine, batch=bsz)
@@ -232,7 +241,7 @@ def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge
             inp["xi"] = rng.uniform(0.05, 3.0, size=inp["pos"].shape).astype(np.float32)
         lse = oracle_lse(inp, wl.n_q_heads, wl.n_kv_heads) if xi_mode == "lse" else None
         gpu = gpu_stage(plan, wl, stage, inp, dtype, xi_mode, lse=lse, kv_mode=kv_mode, paged=paged,
-                        aux_stream=aux_stream, kv_layout=kv_layout)
+                        aux_stream=aux_stream, kv_layout=kv_layout, kv_stream=kv_stream)
         osamp = list(range(bsz)) if oracle_samples is None else oracle_samples
         sub = {key: (val[osamp] if isinstance(val, np.ndarray) and val.shape[:1] == (bsz,) else val)
                for key, val in inp.items()}

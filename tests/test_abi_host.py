@@ -39,7 +39,7 @@ def test_struct_layouts_match_the_header(L, tmp_path):
 int main(void) {
   printf("%zu %zu\\n", sizeof(lightkv_config_t), offsetof(lightkv_config_t, engine));
   printf("%zu %zu\\n", sizeof(lightkv_stage_info_t), offsetof(lightkv_stage_info_t, workspace_bytes));
-  printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, aux_stream));
+  printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, map_event));
   printf("%zu %zu\\n", sizeof(lightkv_kv_args_t), offsetof(lightkv_kv_args_t, stream));
   return 0;
 }
@@ -50,7 +50,7 @@ int main(void) {
     k = L.lightkv
     got = [(C.sizeof(k._Config), k._Config.engine.offset),
            (C.sizeof(k._StageInfo), k._StageInfo.workspace_bytes.offset),
-           (C.sizeof(k._LayerArgs), k._LayerArgs.aux_stream.offset),
+           (C.sizeof(k._LayerArgs), k._LayerArgs.map_event.offset),
            (C.sizeof(k._KvArgs), k._KvArgs.stream.offset)]
     assert got == rows
 

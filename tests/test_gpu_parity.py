@@ -78,6 +78,16 @@ def test_second_stream_inside_compress_layer(name):
         H.run_schedule(S.workload(name), aux_stream=aux)
 
 
+@pytest.mark.parametrize("name", ["small", "cfg1"])
+def test_kv_compaction_behind_the_map_event(name):
+    # lightkv_compact_kv on a second stream behind map_event (recorded once the merge map is complete, before
+    # the hidden-state merge), together with the second stream inside the call
+    import torch
+    aux, kv_stream = torch.cuda.Stream(), torch.cuda.Stream()
+    for _ in range(2):
+        H.run_schedule(S.workload(name), aux_stream=aux, kv_stream=kv_stream)
+
+
 def test_cfg0_fp32_mode():
     H.run_schedule(dataclasses.replace(S.workload("cfg0"), hidden=1024, n_q_heads=8, n_kv_heads=8), dtype="fp32")
 
