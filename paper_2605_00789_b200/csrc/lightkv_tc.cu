@@ -576,14 +576,14 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         cp_async16(sb + t * 4096, p + (bytes ? size_t(kc0) * 128 : 0), bytes);
       }
     };
+    // acc += lo^2 + hi^2 for the four bf16 pairs of v, each product exact in fp32 and added with one rounding
+    // (the mixed-precision fma reads the bf16 halves directly: no unpacking instructions)
     auto sumsq = [](const uint4& v, float acc) {
       const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float lo = __uint_as_float(u[j] << 16), hi = __uint_as_float(u[j] & 0xffff0000u);
-        acc = fmaf(lo, lo, acc);
-        acc = fmaf(hi, hi, acc);
-      }
+      for (int j = 0; j < 4; ++j)
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\t"
+            "fma.rn.f32.bf16 %0, lo, lo, %0;\n\tfma.rn.f32.bf16 %0, hi, hi, %0;\n\t}" : "+f"(acc) : "r"(u[j]));
       return acc;
     };
 
