@@ -202,20 +202,31 @@ def test_selection_over_eight_ctas_ragged_windows():
 
 # ---- full benchmark shapes, compared on the samples the oracle can finish in seconds -----------------
 
+def _bench_streams():
+    # the schedule bench.py times: second stream inside the call (window build and FD beside xi), K/V
+    # compaction on a third stream behind the map event
+    import torch
+    return dict(aux_stream=torch.cuda.Stream(), kv_stream=torch.cuda.Stream())
+
+
 def test_cfg2_full_size_sampled():
-    stats = H.run_schedule(S.workload("cfg2"), oracle_samples=[0, 5])
+    stats = H.run_schedule(S.workload("cfg2"), oracle_samples=[0, 5], **_bench_streams())
     assert [s["n_out"] for s in stats] == [[1440] * 8, [720] * 8, [360] * 8]
 
 
+def test_cfg2_full_size_one_stream():
+    H.run_schedule(S.workload("cfg2"), oracle_samples=[3], stages=[0])
+
+
 def test_cfg3_full_schedule_sampled():
-    stats = H.run_schedule(S.workload("cfg3"), oracle_samples=[0, 31])
+    stats = H.run_schedule(S.workload("cfg3"), oracle_samples=[0, 31], **_bench_streams())
     assert [s["n_out"] for s in stats] == [[288] * 32, [144] * 32, [72] * 32]
 
 
 def test_cfg4_gqa_video_full_schedule_sampled():
     # all three stages: later stages have few large tiles (128 x 128 entries), which the FD kernel splits
     # over clusters of CTAs, and 8192 -> 2048 tokens per sample for the clustered selection kernel
-    stats = H.run_schedule(S.workload("cfg4"), oracle_samples=[1])
+    stats = H.run_schedule(S.workload("cfg4"), oracle_samples=[1], **_bench_streams())
     assert [s["n_out"] for s in stats] == [[4096] * 2, [2048] * 2, [1024] * 2]
 
 
