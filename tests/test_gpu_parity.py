@@ -150,6 +150,20 @@ def test_device_status_word_flags_unsorted_positions():
     assert int(gpu["status"][0]) & 1
 
 
+def test_vanishing_xi_gives_the_group_mean_and_the_status_bit():
+    # xi = 0 for every token of sample 0: the sum over a group vanishes, the merge falls back to the plain
+    # group mean (as the oracle does) and the ZERO_WEIGHT bit is raised; the other samples are unaffected
+    wl = S.workload("small")
+    plan = H.make_plan(wl, xi_mode="given")
+    inp = H.prepare_stage(wl, 0)
+    inp["xi"] = np.random.default_rng(5).uniform(0.05, 3.0, size=inp["pos"].shape).astype(np.float32)
+    inp["xi"][0] = 0.0
+    gpu = H.gpu_stage(plan, wl, 0, inp, xi_mode="given")
+    ref = H.oracle_stage(wl, 0, inp, "given")
+    H.compare_stage(wl, 0, inp, ref, gpu, expect_status=2)
+    plan.close()
+
+
 def test_run_to_run_bit_repeatability():
     wl = S.workload("small")
     plan = H.make_plan(wl)
