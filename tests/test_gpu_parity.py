@@ -214,6 +214,15 @@ def test_selection_over_eight_ctas_ragged_windows():
     assert stats[0]["n_out"][0] < 4480 * 0.6 + 40
 
 
+def test_selection_with_several_tokens_per_thread():
+    # 9600 tokens per sample: more than the 8 x 1024 threads of the largest cluster, so every phase of the
+    # selection kernel loops and its prefix sums take the two-pass path
+    wl = S.Workload(name="sel9600", config_id=121, batch=1, tiles=((100, 96),), n_text=7, hidden=64, n_q_heads=2,
+                    n_kv_heads=2, head_dim=64, n_layers=16, layers=(3, 7, 11), windows=(6, 3, 2),
+                    keep=(0.6, 0.5, 0.7))
+    H.run_schedule(wl, xi_mode="given", stages=[0, 1])
+
+
 # ---- full benchmark shapes, compared on the samples the oracle can finish in seconds -----------------
 
 def _bench_streams():
