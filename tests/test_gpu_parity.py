@@ -254,5 +254,6 @@ def test_cfg4_gqa_video_full_schedule_sampled():
 
 
 def test_cfg4g_large_windows_uniform_xi():
-    # windows of 512 tokens: exercises the multi-chunk B loop of the FD kernels
-    H.run_schedule(S.workload("cfg4g"), xi_mode="uniform", stages=[0], oracle_samples=[0])
+    # windows of 512, 1024 and 2048 tokens: FD tiles of 128 x 128 entries combined across B blocks (atomic
+    # minimum on the keys), the rank loops of the selection kernel over up to 1024 A entries
+    H.run_schedule(S.workload("cfg4g"), xi_mode="uniform", oracle_samples=[0])
