@@ -214,6 +214,17 @@ def test_selection_over_eight_ctas_ragged_windows():
     assert stats[0]["n_out"][0] < 4480 * 0.6 + 40
 
 
+@pytest.mark.parametrize("engine", ["simt", "auto"])
+def test_windows_of_one_and_two_tokens(engine):
+    # a 6 x 8 grid cut 6 x 6: windows of one token (no B node: nothing to merge) and of two (one A, one B);
+    # then 3 x 3 and a single window over what is left
+    wl = S.Workload(name="w12", config_id=122, batch=2, tiles=((6, 8),), n_text=3, hidden=64, n_q_heads=2,
+                    n_kv_heads=1, head_dim=64, n_layers=16, layers=(3, 7, 11), windows=(6, 3, 1),
+                    keep=(0.5, 0.6, 0.5))
+    stats = H.run_schedule(wl, engine=engine)
+    assert stats[0]["n_out"] == [36, 36]          # twelve two-token windows lose one token each
+
+
 def test_selection_with_several_tokens_per_thread():
     # 9600 tokens per sample: more than the 8 x 1024 threads of the largest cluster, so every phase of the
     # selection kernel loops and its prefix sums take the two-pass path
