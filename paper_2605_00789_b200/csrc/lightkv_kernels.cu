@@ -817,10 +817,10 @@ cudaError_t launch_merge_rows(const LayerLaunch& L) {
 // =====================================================================================================
 // K/V merge-compaction ("key and value tokens are compressed simultaneously for later layers").
 // The stage's merge map is applied per KV head; contiguous (strided) or paged (block-table) addressing
-// on either side.  One CTA per output token, small enough in registers for six CTAs per SM; every thread
-// resolves the token's group itself (uniform, cached loads) and keeps the loads of up to four group
-// members in flight per 16-byte unit.  Groups of one are copied; larger groups are summed in fp32 in
-// member order.
+// on either side.  One CTA per output token, five CTAs per SM; every thread resolves the token's group
+// itself (uniform, cached loads) and works on two 16-byte units and two group members at a time, i.e.
+// four loads in flight whatever the group's size (four units on the copy path).  Groups of one are
+// copied; larger groups are summed in fp32 in member order.
 // =====================================================================================================
 struct KvAddr {
   int64_t batch_stride, head_stride, row_stride, page_stride;
