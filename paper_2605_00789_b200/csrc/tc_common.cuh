@@ -1,4 +1,4 @@
-// Inline-PTX building blocks for the sm_100a tensor-core kernels: mbarrier, TMA (no multicast),
+// Inline-PTX building blocks for the sm_100a tensor-core kernels: mbarrier, TMA (one destination CTA per copy),
 // tcgen05 (TMEM allocation, MMA, commit, load), descriptors.  Every wait is bounded.
 #pragma once
 #include <cuda.h>
