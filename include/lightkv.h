@@ -37,7 +37,7 @@
 extern "C" {
 #endif
 
-#define LIGHTKV_VERSION 100
+#define LIGHTKV_VERSION 200
 
 /* status codes */
 #define LIGHTKV_OK               0
@@ -52,7 +52,9 @@ extern "C" {
 #define LIGHTKV_STATUS_POS_ORDER   1u   /* positions not strictly ascending / out of the grid */
 #define LIGHTKV_STATUS_ZERO_WEIGHT 2u   /* a group's xi sum vanished: plain mean was used      */
 #define LIGHTKV_STATUS_TIMEOUT     4u   /* a bounded device-side wait expired                  */
-#define LIGHTKV_STATUS_COUNT       8u   /* n_vis[b] exceeds the stage's capacity               */
+#define LIGHTKV_STATUS_COUNT       8u   /* a sample holds more tokens, A / B nodes or survivors
+                                           than the stage's capacities: its tokens pass through
+                                           unmerged, cut at cap_out                              */
 
 /* storage / arithmetic type of hidden states, Q, K, V */
 #define LIGHTKV_BF16 0   /* bf16 storage, fp32 accumulation                     */
@@ -96,6 +98,14 @@ typedef struct {
   int32_t  dtype;                  /* LIGHTKV_BF16 | LIGHTKV_FP32 */
   int32_t  xi_mode;                /* LIGHTKV_XI_* */
   int32_t  engine;                 /* LIGHTKV_ENGINE_* */
+  int32_t  ragged_input;           /* 0: every sample enters stage 0 with its full grid, so the schedule
+                                         is simulated on the host and capacities are exact wherever the
+                                         counts do not depend on the data.  1: samples may enter with any
+                                         subset of the grid positions (n_vis[b] < cap_in, arbitrary pos):
+                                         every capacity is then an upper bound that holds for any subset,
+                                         cap_a = (cap_in + n_windows) / 2, cap_out = ceil(keep cap_in) +
+                                         n_windows.  A subset given to a plan built with 0 is still safe:
+                                         a sample that overflows a capacity raises LIGHTKV_STATUS_COUNT. */
 } lightkv_config_t;
 
 typedef struct {
@@ -110,6 +120,11 @@ typedef struct {
                                       it entered stage 0 with the full grid (host simulation)     */
   int32_t uses_tensor_cores;       /* 1: the FD and xi contractions of this stage run on tcgen05  */
   size_t  workspace_bytes;         /* DEVICE scratch lightkv_compress_layer needs                 */
+  int32_t cap_a, cap_b;            /* upper bounds on the A / B nodes of one sample               */
+  int32_t fd_tiles;                /* tiles per sample the plan expects the tensor-core FD kernel
+                                      to cut (sizes its launch; the kernel walks whatever tiling
+                                      the device derives from the actual windows)                 */
+  int32_t reserved;
 } lightkv_stage_info_t;
 
 /* Build a plan.  HOST only, no CUDA call.  *out receives the plan.
@@ -133,7 +148,8 @@ typedef struct {
   int32_t  stage;
   int32_t  vis_begin;              /* text rows before the vision block */
   int32_t  n_text_after;           /* rows after it (copied through) */
-  int32_t  text_begin, text_end;   /* prompt-token set J = [text_begin, text_end) within [0, vis_begin] */
+  int32_t  text_begin, text_end;   /* prompt-token set J = [text_begin, text_end) within [0, vis_begin];
+                                      used when n_text_ranges == 0 */
 
   const void* hidden;              /* DEVICE [B, N, d] */
   int64_t hidden_batch_stride, hidden_row_stride;
@@ -184,7 +200,29 @@ typedef struct {
                                       complete, i.e. before the hidden-state merge: lightkv_compact_kv only
                                       needs the map, so a caller may start it on another stream behind this
                                       event, beside the hidden-state merge. */
+  void*   fork_event;              /* cudaEvent_t created by the caller (timing may be disabled); both are */
+  void*   join_event;              /* required with aux_stream (INVALID_ARG otherwise) and unused without it:
+                                      the library records fork_event on `stream` and join_event on
+                                      `aux_stream`, and creates no event of its own.  Once the fork has been
+                                      recorded the join is always enqueued, also when a launch fails. */
+  int32_t n_text_ranges;           /* 0: J = [text_begin, text_end).  1..LIGHTKV_MAX_TEXT_RANGES: J is the union
+                                      of the ranges below */
+  int32_t bidirectional;           /* the causal switch, stored so that a zeroed struct means "causal".
+                                      0: the query at sequence index s sees keys 0..s (a decoder layer).
+                                      1: every query sees all vis_begin + n_vis[b] + n_text_after keys of its
+                                      sample, Eq. "attention-matrix" as printed.  ATTN_LSE must be given the
+                                      log-sum-exp of the same rows. */
+  const int32_t* text_ranges;      /* HOST [n_text_ranges][2]: begin, end of each range; ascending, disjoint,
+                                      inside [0, vis_begin] (copied during the call) */
+  float*  lse_out;                 /* DEVICE [B, H, N] or NULL (ATTN_FULL only): receives, for every vision
+                                      row, the natural-log row log-sum-exp of the scaled (masked) logits the
+                                      xi pass saw -- the quantity ATTN_LSE takes as input, so a caller can
+                                      check its fused attention's own, or feed a later call.  Rows outside
+                                      the vision block are not written. */
+  int64_t lse_out_batch_stride, lse_out_head_stride;
 } lightkv_layer_args_t;
+
+#define LIGHTKV_MAX_TEXT_RANGES 8
 
 #define LIGHTKV_TRACE_EVENTS 6
 

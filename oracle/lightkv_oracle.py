@@ -31,39 +31,60 @@ F64 = np.float64
 # Step 3 (Eq. "attention-factor"): prompt-guidance weight xi
 # --------------------------------------------------------------------------
 
-def attention_rows(q: np.ndarray, k: np.ndarray, vis_begin: int, n_vis: int) -> np.ndarray:
-    """Causal softmax attention rows of the vision queries of one head.
-
-    Eq. "attention-matrix": A = softmax(q K^T / sqrt(d_k)); the decoder is
-    causal, so the query at sequence index s sees keys 0..s.
-    q, k: [N, dh].  Returns A[n_vis, N] (zeros above the diagonal).
-    """
+def scaled_logits(q: np.ndarray, k: np.ndarray, vis_begin: int, n_vis: int, causal: bool = True) -> np.ndarray:
+    """q_i . k_j / sqrt(d_k) for the vision queries of one head, [n_vis, N]; keys a
+    query may not see are set to -inf.  causal: the query at sequence index s
+    sees keys 0..s (a decoder layer); otherwise it sees all N keys."""
     q = np.asarray(q, dtype=F64)
     k = np.asarray(k, dtype=F64)
     n_seq, dh = k.shape
     logits = (q[vis_begin:vis_begin + n_vis] @ k.T) / math.sqrt(dh)
-    s = vis_begin + np.arange(n_vis)[:, None]
-    visible = np.arange(n_seq)[None, :] <= s
-    logits = np.where(visible, logits, -np.inf)
+    if causal:
+        s = vis_begin + np.arange(n_vis)[:, None]
+        logits = np.where(np.arange(n_seq)[None, :] <= s, logits, -np.inf)
+    return logits
+
+
+def attention_rows(q: np.ndarray, k: np.ndarray, vis_begin: int, n_vis: int, causal: bool = True) -> np.ndarray:
+    """Softmax attention rows of the vision queries of one head.
+
+    Eq. "attention-matrix": A = softmax(q K^T / sqrt(d_k)).  The equation prints
+    no mask; the models it is applied to are causal decoders, so the default
+    reading masks keys behind the query (causal=False is the equation as printed).
+    q, k: [N, dh].  Returns A[n_vis, N] (zeros on masked keys).
+    """
+    logits = scaled_logits(q, k, vis_begin, n_vis, causal)
     logits = logits - logits.max(axis=1, keepdims=True)
     e = np.exp(logits)
     return e / e.sum(axis=1, keepdims=True)
 
 
+def row_logsumexp(q: np.ndarray, k: np.ndarray, vis_begin: int, n_vis: int, causal: bool = True) -> np.ndarray:
+    """ln sum_j exp(logit_ij) over the keys query i sees, [n_vis]: the normaliser
+    of Eq. "attention-matrix" that a fused attention kernel keeps per row."""
+    logits = scaled_logits(q, k, vis_begin, n_vis, causal)
+    m = logits.max(axis=1)
+    return m + np.log(np.exp(logits - m[:, None]).sum(axis=1))
+
+
 def xi_from_attention(q: np.ndarray, k: np.ndarray, vis_begin: int, n_vis: int,
-                      text_begin: int, text_end: int) -> np.ndarray:
+                      text_begin: int, text_end: int, causal: bool = True,
+                      text_ranges: Optional[Sequence[Tuple[int, int]]] = None) -> np.ndarray:
     """xi_i = sum_h sum_{j in J} A[h, i, j]  (Eq. "attention-factor").
 
     q: [H, N, dh]; k: [H_kv, N, dh] (query head h reads KV head h // (H / H_kv)).
-    J = [text_begin, text_end) are the prompt-token sequence indices; the sum
-    runs over all H query heads with no averaging, as printed.
+    J = [text_begin, text_end) are the prompt-token sequence indices (or the
+    union of text_ranges when given); the sum runs over all H query heads with
+    no averaging, as printed.
     """
     n_heads, n_kv = q.shape[0], k.shape[0]
     group = n_heads // n_kv
+    ranges = [(text_begin, text_end)] if text_ranges is None else list(text_ranges)
     xi = np.zeros(n_vis, dtype=F64)
     for h in range(n_heads):
-        a = attention_rows(q[h], k[h // group], vis_begin, n_vis)
-        xi += a[:, text_begin:text_end].sum(axis=1)
+        a = attention_rows(q[h], k[h // group], vis_begin, n_vis, causal)
+        for lo, hi in ranges:
+            xi += a[:, lo:hi].sum(axis=1)
     return xi
 
 
@@ -334,7 +355,8 @@ def compress_layer(hidden: np.ndarray, q: Optional[np.ndarray], k: Optional[np.n
                    pos: np.ndarray, n_vis: np.ndarray, vis_begin: int,
                    tiles: Sequence[Tuple[int, int]], w: int, keep: float,
                    text_begin: int = 0, text_end: Optional[int] = None,
-                   xi: Optional[np.ndarray] = None, n_text_after: int = 0
+                   xi: Optional[np.ndarray] = None, n_text_after: int = 0, causal: bool = True,
+                   text_ranges: Optional[Sequence[Tuple[int, int]]] = None
                    ) -> List[Dict[str, np.ndarray]]:
     """One compression stage on a batch (samples are independent).
     hidden [B, N, d]; q [B, H, N, dh]; k [B, H_kv, N, dh]; pos [B, cap]; n_vis [B].
@@ -349,7 +371,8 @@ def compress_layer(hidden: np.ndarray, q: Optional[np.ndarray], k: Optional[np.n
         if xi is not None:
             xi_b = np.asarray(xi[b][:nv], dtype=F64)
         elif q is not None:
-            xi_b = xi_from_attention(q[b][:, :n_seq], k[b][:, :n_seq], vis_begin, nv, text_begin, text_end)
+            xi_b = xi_from_attention(q[b][:, :n_seq], k[b][:, :n_seq], vis_begin, nv, text_begin, text_end,
+                                     causal, text_ranges)
         else:
             xi_b = np.ones(nv, dtype=F64)
         res = compress_sequence(hidden[b][:n_seq], vis_begin, nv, pos[b][:nv], xi_b, tiles, w, keep)

@@ -11,6 +11,7 @@ namespace lkv {
 constexpr int kMaxTiles = 32;          // image tiles / frames per sample
 constexpr int kFdTile = 128;           // A (and B) entries per tile of the tensor-core FD kernel
 constexpr int kMaxWindows = 2048;      // windows per sample (window-build kernel keeps 32 x n_windows u16 counters in smem)
+constexpr int kMaxWindowTokens = 65535;  // tokens of one window (range of those counters)
 
 // Grid geometry of one stage, passed by value to the kernels.
 struct Geometry {
@@ -55,6 +56,28 @@ struct Workspace {
   int* slot;       // [B, cap_in]         output slot of surviving tokens
   int* a_partner;  // [B, cap_a]          per A entry: token it is merged into, -1 = survives
   int cap_in, cap_out, cap_a, cap_b, n_windows;
+};
+
+// Prompt-token set J: up to LIGHTKV_MAX_TEXT_RANGES ascending, disjoint ranges of sequence indices in front of
+// the vision block.  begin / end bound the whole set.
+struct TextSet {
+  int n;
+  int begin, end;
+  int lo[LIGHTKV_MAX_TEXT_RANGES], hi[LIGHTKV_MAX_TEXT_RANGES];
+  __host__ __device__ inline bool holds(int j) const {
+    for (int i = 0; i < n; ++i)
+      if (j >= lo[i] && j < hi[i]) return true;
+    return false;
+  }
+  // bit c set <=> key j0 + c belongs to J (c < 64)
+  __host__ __device__ inline unsigned long long mask64(int j0) const {
+    unsigned long long m = 0;
+    for (int i = 0; i < n; ++i) {
+      const int a = (lo[i] > j0 ? lo[i] : j0) - j0, b = (hi[i] < j0 + 64 ? hi[i] : j0 + 64) - j0;
+      if (b > a) m |= (b - a >= 64 ? ~0ull : ((1ull << (b - a)) - 1ull)) << a;
+    }
+    return m;
+  }
 };
 
 // Tokens removed from a window of n tokens when a fraction `keep` must remain:

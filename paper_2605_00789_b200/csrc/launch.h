@@ -1,5 +1,7 @@
 // Host-side launch interface between the C ABI (lightkv_api.cu) and the kernel files.
 #pragma once
+#include <mutex>
+
 #include "common.cuh"
 
 namespace lkv {
@@ -36,9 +38,34 @@ struct LayerLaunch {
   int fd_tiles;                      // estimate of FdTiling::n_tiles per sample (launch shape of the tensor-core FD kernel)
   Geometry geo;
   Workspace ws;
+  TextSet text;                      // prompt-token set J of this call
   const lightkv_layer_args_t* a;
   cudaStream_t stream;
 };
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per (kernel, device) instead of before every launch.
+struct SmemAttrEntry { const void* kernel; int dev; int bytes; };
+inline cudaError_t ensure_dynamic_smem_ptr(const void* kernel, int bytes) {
+  static std::mutex mu;
+  static SmemAttrEntry table[64];
+  static int used = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  SmemAttrEntry* e = nullptr;
+  for (int i = 0; i < used; ++i)
+    if (table[i].kernel == kernel && table[i].dev == dev) { e = &table[i]; break; }
+  if (e && e->bytes >= bytes) return cudaSuccess;
+  const cudaError_t rc = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (rc != cudaSuccess) return rc;
+  if (!e && used < 64) e = &table[used++];
+  if (e) { e->kernel = kernel; e->dev = dev; e->bytes = bytes; }
+  return cudaSuccess;
+}
+template <typename... P>
+inline cudaError_t ensure_dynamic_smem(void (*kernel)(P...), int bytes) {
+  return ensure_dynamic_smem_ptr(reinterpret_cast<const void*>(kernel), bytes);
+}
 
 // window build (Step 1 and "Window partitioning")
 cudaError_t launch_window_build(const LayerLaunch& L);

@@ -118,6 +118,7 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
   if (c->dtype != LIGHTKV_BF16 && c->dtype != LIGHTKV_FP32) return LIGHTKV_ERR_INVALID_ARG;
   if (c->xi_mode < LIGHTKV_XI_GIVEN || c->xi_mode > LIGHTKV_XI_UNIFORM) return LIGHTKV_ERR_INVALID_ARG;
   if (c->engine != LIGHTKV_ENGINE_AUTO && c->engine != LIGHTKV_ENGINE_SIMT) return LIGHTKV_ERR_INVALID_ARG;
+  if (c->ragged_input != 0 && c->ragged_input != 1) return LIGHTKV_ERR_INVALID_ARG;
   if (c->n_tiles > kMaxTiles) return LIGHTKV_ERR_UNSUPPORTED;
   if (c->head_dim > 256) return LIGHTKV_ERR_UNSUPPORTED;
 
@@ -138,7 +139,7 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
   // the surviving positions do not depend on the data and the counts are exact.
   std::vector<int> alive(p->n_vis0);
   for (int i = 0; i < p->n_vis0; ++i) alive[i] = i;
-  bool exact = true;
+  bool exact = c->ragged_input == 0;   // a subset of the grid makes every later count depend on the data
   int cap = p->n_vis0;
   for (int s = 0; s < c->n_stages; ++s) {
     StagePlan sp;
@@ -155,6 +156,12 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
       g.tile_off[t + 1] = g.tile_off[t] + g.rows[t] * g.cols[t];
     }
     if (g.n_windows > kMaxWindows) { delete p; return LIGHTKV_ERR_UNSUPPORTED; }
+    // the window-build kernel counts the tokens of a window in 16 bits
+    for (int t = 0; t < c->n_tiles; ++t)
+      if ((long long)((g.rows[t] + sp.w - 1) / sp.w) * ((g.cols[t] + sp.w - 1) / sp.w) > kMaxWindowTokens) {
+        delete p;
+        return LIGHTKV_ERR_UNSUPPORTED;
+      }
     sp.n_windows = g.n_windows;
     sp.cap_in = cap;
     sp.exact = exact;
@@ -220,6 +227,7 @@ int lightkv_plan_stage_info(const lightkv_plan_t* p, int32_t stage, lightkv_stag
                                             p->cfg.xi_mode == LIGHTKV_XI_ATTN_LSE) &&
                                            tc_xi_supported(p->cfg.head_dim)))) ? 1 : 0;
   info->workspace_bytes = s.ws_bytes;
+  info->cap_a = s.cap_a; info->cap_b = s.cap_b; info->fd_tiles = s.fd_tiles; info->reserved = 0;
   return LIGHTKV_OK;
 }
 
@@ -248,7 +256,25 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
   const size_t esz = c.dtype == LIGHTKV_BF16 ? 2 : 4;
   if (a->vis_begin < 0 || a->n_text_after < 0 || a->vis_begin + a->n_text_after > c.max_text)
     return LIGHTKV_ERR_INVALID_ARG;
-  if (a->text_begin < 0 || a->text_end < a->text_begin || a->text_end > a->vis_begin) return LIGHTKV_ERR_INVALID_ARG;
+  TextSet text;
+  memset(&text, 0, sizeof(text));
+  if (a->n_text_ranges < 0 || a->n_text_ranges > LIGHTKV_MAX_TEXT_RANGES) return LIGHTKV_ERR_INVALID_ARG;
+  if (a->n_text_ranges == 0) {
+    if (a->text_begin < 0 || a->text_end < a->text_begin || a->text_end > a->vis_begin) return LIGHTKV_ERR_INVALID_ARG;
+    text.n = 1; text.lo[0] = a->text_begin; text.hi[0] = a->text_end;
+  } else {
+    if (!a->text_ranges) return LIGHTKV_ERR_INVALID_ARG;
+    int prev_end = 0;
+    for (int i = 0; i < a->n_text_ranges; ++i) {
+      const int lo = a->text_ranges[2 * i], hi = a->text_ranges[2 * i + 1];
+      if (lo < prev_end || hi < lo || hi > a->vis_begin) return LIGHTKV_ERR_INVALID_ARG;   // ascending, disjoint
+      text.lo[i] = lo; text.hi[i] = hi;
+      prev_end = hi;
+    }
+    text.n = a->n_text_ranges;
+  }
+  text.begin = text.lo[0]; text.end = text.hi[text.n - 1];
+  if (a->bidirectional != 0 && a->bidirectional != 1) return LIGHTKV_ERR_INVALID_ARG;
   if (!a->hidden || !a->hidden_out || !a->n_vis_out || !a->pos_out || !a->dst || !a->weight || !a->grp_off ||
       !a->grp_src || !a->workspace)
     return LIGHTKV_ERR_INVALID_ARG;
@@ -271,12 +297,14 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
     if (c.xi_mode == LIGHTKV_XI_ATTN_LSE && !a->lse) return LIGHTKV_ERR_INVALID_ARG;
   }
   if (c.xi_mode == LIGHTKV_XI_GIVEN && !a->xi) return LIGHTKV_ERR_INVALID_ARG;
+  if (a->lse_out && c.xi_mode != LIGHTKV_XI_ATTN_FULL) return LIGHTKV_ERR_INVALID_ARG;
+  if (a->aux_stream && (!a->fork_event || !a->join_event)) return LIGHTKV_ERR_INVALID_ARG;
 
   LayerLaunch L;
   L.batch = c.batch; L.hidden = c.hidden; L.n_q_heads = c.n_q_heads; L.n_kv_heads = c.n_kv_heads;
   L.head_dim = c.head_dim; L.dtype = c.dtype; L.xi_mode = c.xi_mode; L.keep = s.keep; L.geo = s.geo;
   L.fd_tiles = s.fd_tiles;
-  L.ws = bind_workspace(s, a->workspace); L.a = a; L.stream = static_cast<cudaStream_t>(a->stream);
+  L.ws = bind_workspace(s, a->workspace); L.text = text; L.a = a; L.stream = static_cast<cudaStream_t>(a->stream);
 
   cudaEvent_t* ev = reinterpret_cast<cudaEvent_t*>(a->trace_events);
   auto mark = [&](int i) { return ev ? cudaEventRecord(ev[i], L.stream) : cudaSuccess; };
@@ -284,24 +312,19 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
   const bool tc_fd = s.use_tc && tc_fd_supported(c.hidden);
   cudaStream_t aux = (a->aux_stream && attn && !ev) ? static_cast<cudaStream_t>(a->aux_stream) : nullptr;
   if (aux) {
-    // fork: window build + FD (HBM bound) on the second stream, xi (bound by the exponentials) on the first
-    cudaEvent_t fork = nullptr, join = nullptr;
-    if (cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) != cudaSuccess) return LIGHTKV_ERR_CUDA;
-    if (cudaEventCreateWithFlags(&join, cudaEventDisableTiming) != cudaSuccess) {
-      cudaEventDestroy(fork);
-      return LIGHTKV_ERR_CUDA;
-    }
+    // fork: window build + FD (HBM bound) on the second stream, xi (bound by the exponentials) on the first.
+    // The events are the caller's; once the fork is recorded the join is enqueued whatever happens between.
+    cudaEvent_t fork = static_cast<cudaEvent_t>(a->fork_event), join = static_cast<cudaEvent_t>(a->join_event);
     LayerLaunch La = L;
     La.stream = aux;
-    bool ok = cudaEventRecord(fork, L.stream) == cudaSuccess && cudaStreamWaitEvent(aux, fork, 0) == cudaSuccess;
+    if (cudaEventRecord(fork, L.stream) != cudaSuccess) return LIGHTKV_ERR_CUDA;
+    bool ok = cudaStreamWaitEvent(aux, fork, 0) == cudaSuccess;
     ok = ok && launch_window_build(La) == cudaSuccess;
     ok = ok && (tc_fd ? launch_fd_tc(La) : launch_fd_simt(La)) == cudaSuccess;
-    ok = ok && cudaEventRecord(join, aux) == cudaSuccess;
+    const bool joined = cudaEventRecord(join, aux) == cudaSuccess;
     ok = ok && (tc_xi ? launch_xi_tc(L) : launch_xi_simt(L)) == cudaSuccess;
-    ok = ok && cudaStreamWaitEvent(L.stream, join, 0) == cudaSuccess;
-    cudaEventDestroy(fork);                 // released once the recorded work has completed
-    cudaEventDestroy(join);
-    if (!ok) return LIGHTKV_ERR_CUDA;
+    const bool waited = joined && cudaStreamWaitEvent(L.stream, join, 0) == cudaSuccess;
+    if (!ok || !waited) return LIGHTKV_ERR_CUDA;
   } else {
     if (mark(0) != cudaSuccess) return LIGHTKV_ERR_CUDA;
     if (launch_window_build(L) != cudaSuccess || mark(1) != cudaSuccess) return LIGHTKV_ERR_CUDA;

@@ -98,9 +98,14 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
     if (lane == 31) { wsum[nW] = xs; asum[nW] = xa; }
   }
   __syncthreads();
+  // A sample whose A or B nodes do not fit the plan's capacities (a subset of the grid handed to a plan that was
+  // built for full grids) keeps all of its tokens: its windows are published empty, so no later kernel finds an
+  // entry, a tile or a window size for it, nothing is indexed past a row, and the status word says so.
+  const bool over = asum[nW] > ws.cap_a || wsum[nW] - asum[nW] > ws.cap_b;
+  if (over && tid == 0) set_status(status, LIGHTKV_STATUS_COUNT);
   for (int w = tid; w <= nW; w += blockDim.x) {
-    ws.win_off[size_t(b) * (nW + 1) + w] = wsum[w];
-    ws.a_off[size_t(b) * (nW + 1) + w] = asum[w];
+    ws.win_off[size_t(b) * (nW + 1) + w] = over ? 0 : wsum[w];
+    ws.a_off[size_t(b) * (nW + 1) + w] = over ? 0 : asum[w];
   }
   {  // largest A and B side of any window -> tiling of the tensor-core FD kernel
     int ma = 0, mb = 0;
@@ -130,7 +135,7 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
           t.blocks_a = (ma + kFdTile - 1) / kFdTile; t.blocks_b = (mb + kFdTile - 1) / kFdTile;
           t.passes = 4;
         }
-        t.n_tiles = (mb > 0) ? ((nW + t.wpt - 1) / t.wpt) * t.blocks_a * t.blocks_b : 0;
+        t.n_tiles = (mb > 0 && !over) ? ((nW + t.wpt - 1) / t.wpt) * t.blocks_a * t.blocks_b : 0;
         t.pad[0] = t.pad[1] = t.pad[2] = 0;
         ws.fd_tiling[b] = t;
       }
@@ -166,8 +171,7 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
 cudaError_t launch_window_build(const LayerLaunch& L) {
   const int nW = L.geo.n_windows;
   const size_t smem = ((size_t(32) * nW * 2 + 15) & ~size_t(15)) + size_t(2) * (nW + 1) * sizeof(int);
-  cudaError_t e = cudaFuncSetAttribute(window_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       200 * 1024);
+  const cudaError_t e = ensure_dynamic_smem(window_build_kernel, 200 * 1024);
   if (e != cudaSuccess) return e;
   return launch_kernel(window_build_kernel, L.batch, 1024, smem, L.stream, 1, L.geo, L.a->pos, L.a->n_vis, L.ws, L.a->status);
 }
@@ -321,32 +325,42 @@ cudaError_t launch_fd_simt(const LayerLaunch& L) {
 constexpr int XI_TQ = 32, XI_TK = 64;
 
 template <typename T>
+struct XiSimtArgs {
+  const T* q; int64_t q_bs, q_hs, q_rs;
+  const T* k; int64_t k_bs, k_hs, k_rs;
+  const float* lse; int64_t lse_bs, lse_hs;        // caller's row log-sum-exp (ATTN_LSE) or nullptr
+  float* lse_out; int64_t lse_out_bs, lse_out_hs;  // receives the row log-sum-exp (ATTN_FULL) or nullptr
+  const int* n_vis;
+  int vis_begin, n_text_after, bidirectional;
+  int n_q_heads, n_kv_heads, dh;
+  TextSet text;
+};
+
+template <typename T>
 __global__ void __launch_bounds__(256)
-xi_simt_kernel(const T* __restrict__ q, int64_t q_bs, int64_t q_hs, int64_t q_rs,
-               const T* __restrict__ k, int64_t k_bs, int64_t k_hs, int64_t k_rs,
-               const float* __restrict__ lse, int64_t lse_bs, int64_t lse_hs,
-               const int* __restrict__ n_vis, int vis_begin, int text_begin, int text_end,
-               int n_q_heads, int n_kv_heads, int dh, Workspace ws) {
+xi_simt_kernel(XiSimtArgs<T> a, Workspace ws) {
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int ld = dh + 1;
+  const int dh = a.dh, ld = dh + 1;
   float* Qs = reinterpret_cast<float*>(smem_raw);       // [XI_TQ][ld]
   float* Ks = Qs + XI_TQ * ld;                          // [XI_TK][ld]
   float* Ss = Ks + XI_TK * ld;                          // [XI_TQ][XI_TK + 1]
 
   const int b = blockIdx.z, h = blockIdx.y, t0 = blockIdx.x * XI_TQ, tid = threadIdx.x;
-  int n = n_vis ? min(n_vis[b], ws.cap_in) : ws.cap_in;
+  int n = a.n_vis ? min(a.n_vis[b], ws.cap_in) : ws.cap_in;
   if (t0 >= n) return;
   const int nq = min(XI_TQ, n - t0);
-  const int hk = h / (n_q_heads / n_kv_heads);
-  const T* qh = q + size_t(b) * q_bs + size_t(h) * q_hs;
-  const T* kh = k + size_t(b) * k_bs + size_t(hk) * k_hs;
+  const int hk = h / (a.n_q_heads / a.n_kv_heads);
+  const T* qh = a.q + size_t(b) * a.q_bs + size_t(h) * a.q_hs;
+  const T* kh = a.k + size_t(b) * a.k_bs + size_t(hk) * a.k_hs;
   const float scale2 = 1.4426950408889634f / sqrtf((float)dh);      // logits in log2 units
+  const int vis_begin = a.vis_begin;
+  const int n_seq = vis_begin + n + a.n_text_after;                   // keys of this sample
 
   for (int idx = tid; idx < XI_TQ * (dh / 4); idx += blockDim.x) {
     const int r = idx / (dh / 4), c = (idx % (dh / 4)) * 4;
     float f[4] = {0.f, 0.f, 0.f, 0.f};
-    if (r < nq) load4<T>(qh + size_t(vis_begin + t0 + r) * q_rs + c, f);
+    if (r < nq) load4<T>(qh + size_t(vis_begin + t0 + r) * a.q_rs + c, f);
 #pragma unroll
     for (int j = 0; j < 4; ++j) Qs[r * ld + c + j] = f[j];
   }
@@ -357,9 +371,10 @@ xi_simt_kernel(const T* __restrict__ q, int64_t q_bs, int64_t q_hs, int64_t q_rs
 #pragma unroll
   for (int i = 0; i < 4; ++i) { m_run[i] = -INFINITY; l_all[i] = 0.f; l_txt[i] = 0.f; }
 
-  const int s_last = vis_begin + t0 + nq - 1;           // last key any row of the tile may see
-  const int key_lo = lse ? text_begin : 0;
-  const int key_hi = lse ? min(text_end, s_last + 1) : s_last + 1;
+  // last key any row of the tile may see: its own (causal) or the sample's last (bidirectional)
+  const int s_last = a.bidirectional ? n_seq - 1 : vis_begin + t0 + nq - 1;
+  const int key_lo = a.lse ? a.text.begin : 0;
+  const int key_hi = a.lse ? min(a.text.end, s_last + 1) : s_last + 1;
 
   for (int j0 = key_lo; j0 < key_hi; j0 += XI_TK) {
     const int nk = min(XI_TK, key_hi - j0);
@@ -367,7 +382,7 @@ xi_simt_kernel(const T* __restrict__ q, int64_t q_bs, int64_t q_hs, int64_t q_rs
     for (int idx = tid; idx < XI_TK * (dh / 4); idx += blockDim.x) {
       const int r = idx / (dh / 4), c = (idx % (dh / 4)) * 4;
       float f[4] = {0.f, 0.f, 0.f, 0.f};
-      if (r < nk) load4<T>(kh + size_t(j0 + r) * k_rs + c, f);
+      if (r < nk) load4<T>(kh + size_t(j0 + r) * a.k_rs + c, f);
 #pragma unroll
       for (int j = 0; j < 4; ++j) Ks[r * ld + c + j] = f[j];
     }
@@ -387,22 +402,24 @@ xi_simt_kernel(const T* __restrict__ q, int64_t q_bs, int64_t q_hs, int64_t q_rs
 #pragma unroll
       for (int j = 0; j < 4; ++j) Ss[(2 * ty + i) * (XI_TK + 1) + 4 * tx + j] = acc[i][j] * scale2;
     __syncthreads();
+    const unsigned long long tmask = a.text.mask64(j0);      // XI_TK = 64 columns
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int r = 4 * wp + i;
       if (r >= nq) continue;                            // warp-uniform
       const int s_i = vis_begin + t0 + r;
+      const int last = a.bidirectional ? n_seq - 1 : s_i;
       float v[2];
       bool ok[2], txt[2];
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int j = j0 + lane + 32 * c;
-        ok[c] = (lane + 32 * c < nk) && j <= s_i;
-        txt[c] = ok[c] && j >= text_begin && j < text_end;
+        ok[c] = (lane + 32 * c < nk) && j <= last;
+        txt[c] = ok[c] && ((tmask >> (lane + 32 * c)) & 1ull);
         v[c] = ok[c] ? Ss[r * (XI_TK + 1) + lane + 32 * c] : -INFINITY;
       }
-      if (lse) {
-        const float l2 = lse[size_t(b) * lse_bs + size_t(h) * lse_hs + s_i] * 1.4426950408889634f;
+      if (a.lse) {
+        const float l2 = a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_i] * 1.4426950408889634f;
         float p = (txt[0] ? exp2f(v[0] - l2) : 0.f) + (txt[1] ? exp2f(v[1] - l2) : 0.f);
         for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
         l_txt[i] += p;
@@ -427,39 +444,37 @@ xi_simt_kernel(const T* __restrict__ q, int64_t q_bs, int64_t q_hs, int64_t q_rs
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int r = 4 * wp + i;
-      if (r < nq)
-        ws.xi_h[(size_t(b) * n_q_heads + h) * ws.cap_in + t0 + r] = lse ? l_txt[i] : l_txt[i] / l_all[i];
+      if (r < nq) {
+        ws.xi_h[(size_t(b) * a.n_q_heads + h) * ws.cap_in + t0 + r] = a.lse ? l_txt[i] : l_txt[i] / l_all[i];
+        if (a.lse_out)
+          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + vis_begin + t0 + r] =
+              (m_run[i] + log2f(l_all[i])) * 0.6931471805599453f;
+      }
     }
   }
 }
 
-cudaError_t launch_xi_simt(const LayerLaunch& L) {
+template <typename T>
+static cudaError_t launch_xi_simt_t(const LayerLaunch& L) {
   const lightkv_layer_args_t* a = L.a;
   const int dh = L.head_dim;
   const size_t smem = (size_t(XI_TQ + XI_TK) * (dh + 1) + size_t(XI_TQ) * (XI_TK + 1)) * sizeof(float);
   const dim3 grid((L.ws.cap_in + XI_TQ - 1) / XI_TQ, L.n_q_heads, L.batch);
-  const float* lse = L.xi_mode == LIGHTKV_XI_ATTN_LSE ? a->lse : nullptr;
-  cudaError_t e;
-  if (L.dtype == LIGHTKV_BF16) {
-    auto kern = xi_simt_kernel<__nv_bfloat16>;
-    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024)) != cudaSuccess)
-      return e;
-    return launch_kernel(kern, grid, 256, smem, L.stream, 1,
-        static_cast<const __nv_bfloat16*>(a->q), a->q_batch_stride, a->q_head_stride, a->q_row_stride,
-        static_cast<const __nv_bfloat16*>(a->k), a->k_batch_stride, a->k_head_stride, a->k_row_stride,
-        lse, a->lse_batch_stride, a->lse_head_stride, a->n_vis, a->vis_begin, a->text_begin, a->text_end,
-        L.n_q_heads, L.n_kv_heads, dh, L.ws);
-  } else {
-    auto kern = xi_simt_kernel<float>;
-    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024)) != cudaSuccess)
-      return e;
-    return launch_kernel(kern, grid, 256, smem, L.stream, 1,
-        static_cast<const float*>(a->q), a->q_batch_stride, a->q_head_stride, a->q_row_stride,
-        static_cast<const float*>(a->k), a->k_batch_stride, a->k_head_stride, a->k_row_stride,
-        lse, a->lse_batch_stride, a->lse_head_stride, a->n_vis, a->vis_begin, a->text_begin, a->text_end,
-        L.n_q_heads, L.n_kv_heads, dh, L.ws);
-  }
-  return cudaGetLastError();
+  XiSimtArgs<T> x;
+  x.q = static_cast<const T*>(a->q); x.q_bs = a->q_batch_stride; x.q_hs = a->q_head_stride; x.q_rs = a->q_row_stride;
+  x.k = static_cast<const T*>(a->k); x.k_bs = a->k_batch_stride; x.k_hs = a->k_head_stride; x.k_rs = a->k_row_stride;
+  x.lse = L.xi_mode == LIGHTKV_XI_ATTN_LSE ? a->lse : nullptr; x.lse_bs = a->lse_batch_stride; x.lse_hs = a->lse_head_stride;
+  x.lse_out = L.xi_mode == LIGHTKV_XI_ATTN_FULL ? a->lse_out : nullptr;
+  x.lse_out_bs = a->lse_out_batch_stride; x.lse_out_hs = a->lse_out_head_stride;
+  x.n_vis = a->n_vis; x.vis_begin = a->vis_begin; x.n_text_after = a->n_text_after; x.bidirectional = a->bidirectional;
+  x.n_q_heads = L.n_q_heads; x.n_kv_heads = L.n_kv_heads; x.dh = dh; x.text = L.text;
+  const cudaError_t e = ensure_dynamic_smem(xi_simt_kernel<T>, 160 * 1024);
+  if (e != cudaSuccess) return e;
+  return launch_kernel(xi_simt_kernel<T>, grid, 256, smem, L.stream, 1, x, L.ws);
+}
+
+cudaError_t launch_xi_simt(const LayerLaunch& L) {
+  return L.dtype == LIGHTKV_BF16 ? launch_xi_simt_t<__nv_bfloat16>(L) : launch_xi_simt_t<float>(L);
 }
 
 // =====================================================================================================

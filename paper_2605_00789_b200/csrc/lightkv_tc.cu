@@ -70,7 +70,11 @@ struct XiTcArgs {
   uint32_t* status;
   const float* lse;                  // [B, H, N] row log-sum-exp (natural log) from the caller, or nullptr
   int64_t lse_bs, lse_hs;
-  int cap_in, vis_begin, text_begin, text_end, n_q_heads, group;
+  float* lse_out;                    // [B, H, N] receives the row log-sum-exp of the vision rows, or nullptr
+  int64_t lse_out_bs, lse_out_hs;
+  TextSet text;                      // prompt-token set J
+  int n_text_after, bidirectional;   // bidirectional: every query sees all keys of its sample
+  int cap_in, vis_begin, n_q_heads, group;
   int batch, n_qt;                   // samples, query tiles of 128 rows per (sample, head)
   float scale2;                      // log2(e) / sqrt(dh)
 };
@@ -109,9 +113,9 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   const int n_items = WALK ? a.n_qt * a.n_q_heads * a.batch : 0;
   // key tiles to visit: all tiles up to the last query's own key, or, when the caller supplies the row
   // log-sum-exp, only the tiles that hold prompt keys (J lies before the vision block, so it is visible)
-  const int kt_lo = a.lse ? a.text_begin / BK : 0;
-  const int nkt_lse = a.text_end > a.text_begin ? (a.text_end - 1) / BK + 1 - kt_lo : 0;
-  struct Item { int h, b, t0, nq, s_first, nkt; };
+  const int kt_lo = a.lse ? a.text.begin / BK : 0;
+  const int nkt_lse = a.text.end > a.text.begin ? (a.text.end - 1) / BK + 1 - kt_lo : 0;
+  struct Item { int h, b, t0, nq, s_first, nkt, n_seq; };
   auto decode = [&](int item, Item& it) -> bool {
     int qt;
     if (WALK) {
@@ -125,7 +129,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     if (it.t0 >= n) return false;
     it.nq = min(128, n - it.t0);
     it.s_first = a.vis_begin + it.t0;
-    it.nkt = a.lse ? nkt_lse : (it.s_first + it.nq - 1) / BK + 1;
+    it.n_seq = a.vis_begin + n + a.n_text_after;
+    it.nkt = a.lse ? nkt_lse : ((a.bidirectional ? it.n_seq : it.s_first + it.nq) - 1) / BK + 1;
     return true;
   };
   Item it0 = {};
@@ -228,22 +233,23 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
 
         if (a.lse) {                                      // normaliser known: only the prompt columns count
           const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
-          const int lo = a.text_begin - j0, hi = a.text_end - j0;
+          const unsigned long long tm = a.text.mask64(j0);     // BK <= 64 columns
           float st = 0.f;
 #pragma unroll
           for (int c = 0; c < NC; ++c)
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (c * 32 + i >= lo && c * 32 + i < hi) st += ex2(fmaf(v[c][i], sc, -l2));
+              if ((tm >> (c * 32 + i)) & 1ull) st += ex2(fmaf(v[c][i], sc, -l2));
           l_txt += st;
           l_all = 1.f;
           continue;
         }
-        const bool in_j = j0 < a.text_end && j0 + BK > a.text_begin;   // tile reaches into the prompt set J
-        if (j0 + BK - 1 > s_first) {
-          // ---- tile straddles the diagonal: causal mask.  Columns beyond the warp's last visible one are skipped
-          // in blocks of eight (a warp-uniform test), so most of the masked half costs no exponentials.
-          const int lim = s_first + r - j0;               // last visible column of this row (may be negative)
+        const bool in_j = j0 < a.text.end && j0 + BK > a.text.begin;   // tile reaches into the prompt set J
+        if (j0 + BK - 1 > (a.bidirectional ? it.n_seq - 1 : s_first)) {
+          // ---- tile straddles the diagonal (or, without the causal mask, the end of the sample): mask.  Columns
+          // beyond the warp's last visible one are skipped in blocks of eight (a warp-uniform test), so most of
+          // the masked half costs no exponentials.
+          const int lim = (a.bidirectional ? it.n_seq - 1 : s_first + r) - j0;   // last visible column of this row (may be negative)
           const int lim_max = __reduce_max_sync(0xffffffffu, lim);
           if (lim_max < 0) continue;                      // no row of this warp sees any key of the tile
 #pragma unroll
@@ -294,14 +300,14 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         const float ms = m_new * sc;
         float sa = 0.f, st = 0.f;
         if (in_j) {
-          const int lo = a.text_begin - j0, hi = a.text_end - j0;
+          const unsigned long long tm = a.text.mask64(j0);     // BK <= 64 columns
 #pragma unroll
           for (int c = 0; c < NC; ++c)
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const float p = ex2(fmaf(v[c][i], sc, -ms));
               sa += p;
-              if (c * 32 + i >= lo && c * 32 + i < hi) st += p;
+              if ((tm >> (c * 32 + i)) & 1ull) st += p;
             }
         } else {
           float part[NC];                                   // independent sums
@@ -319,8 +325,12 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         l_txt = fmaf(l_txt, resc, st);
         m_run = m_new;
       }
-      if (alive && r < nq && !*abort_flag)
+      if (alive && r < nq && !*abort_flag) {
         a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + it.t0 + r] = a.lse ? l_txt : l_txt / l_all;
+        if (a.lse_out)
+          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + s_first + r] =
+              fmaf(m_run, sc, log2f(l_all)) * 0.6931471805599453f;
+      }
       if (!WALK) break;
     }
   }
@@ -349,7 +359,10 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   XiTcArgs x;
   x.n_vis = a->n_vis; x.xi_h = L.ws.xi_h; x.status = a->status; x.cap_in = L.ws.cap_in;
   x.lse = L.xi_mode == LIGHTKV_XI_ATTN_LSE ? a->lse : nullptr; x.lse_bs = a->lse_batch_stride; x.lse_hs = a->lse_head_stride;
-  x.vis_begin = a->vis_begin; x.text_begin = a->text_begin; x.text_end = a->text_end;
+  x.lse_out = L.xi_mode == LIGHTKV_XI_ATTN_FULL ? a->lse_out : nullptr;
+  x.lse_out_bs = a->lse_out_batch_stride; x.lse_out_hs = a->lse_out_head_stride;
+  x.text = L.text; x.n_text_after = a->n_text_after; x.bidirectional = a->bidirectional;
+  x.vis_begin = a->vis_begin;
   x.n_q_heads = L.n_q_heads; x.group = L.n_q_heads / L.n_kv_heads;
   x.scale2 = 1.4426950408889634f / sqrtf((float)L.head_dim);
   x.batch = L.batch; x.n_qt = (L.ws.cap_in + 127) / 128;
@@ -365,7 +378,7 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   constexpr int BK = XT_KEY_TILE;
   const size_t smem = size_t(L.head_dim / 64) * (16384 + size_t(XT_STAGES) * BK * 128) + 1024 + 256;
   auto launch = [&](auto kernel) -> cudaError_t {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = ensure_dynamic_smem(kernel, (int)smem);
     if (e != cudaSuccess) return e;
     return launch_kernel(kernel, grid, 192, smem, L.stream, 1, qm, km, x);
   };
@@ -795,12 +808,10 @@ cudaError_t launch_fd_tc(const LayerLaunch& L) {
   const int clusters = (int)std::min<long long>(bound, slots / ks);
   cudaError_t e;
   if (ks == 1) {
-    if ((e = cudaFuncSetAttribute(fd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM)) != cudaSuccess)
-      return e;
+    if ((e = ensure_dynamic_smem(fd_tc_kernel<false>, (int)FT_SMEM)) != cudaSuccess) return e;
     return launch_kernel(fd_tc_kernel<false>, clusters, FT_LOADERS + 32, FT_SMEM, L.stream, 1, f);
   }
-  if ((e = cudaFuncSetAttribute(fd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM)) != cudaSuccess)
-    return e;
+  if ((e = ensure_dynamic_smem(fd_tc_kernel<true>, (int)FT_SMEM)) != cudaSuccess) return e;
   return launch_kernel(fd_tc_kernel<true>, clusters * ks, FT_LOADERS + 32, FT_SMEM, L.stream, ks, f);
 }
 

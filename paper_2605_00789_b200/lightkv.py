@@ -33,14 +33,15 @@ class _Config(C.Structure):
                 ("n_stages", C.c_int32), ("layers", C.POINTER(C.c_int32)),
                 ("windows", C.POINTER(C.c_int32)), ("keep", C.POINTER(C.c_double)),
                 ("max_text", C.c_int32), ("dtype", C.c_int32), ("xi_mode", C.c_int32),
-                ("engine", C.c_int32)]
+                ("engine", C.c_int32), ("ragged_input", C.c_int32)]
 
 
 class _StageInfo(C.Structure):
     _fields_ = [("layer", C.c_int32), ("window", C.c_int32), ("keep", C.c_double),
                 ("cap_in", C.c_int32), ("cap_out", C.c_int32), ("n_windows", C.c_int32),
                 ("counts_exact", C.c_int32), ("uses_tensor_cores", C.c_int32),
-                ("workspace_bytes", C.c_size_t)]
+                ("workspace_bytes", C.c_size_t), ("cap_a", C.c_int32), ("cap_b", C.c_int32),
+                ("fd_tiles", C.c_int32), ("reserved", C.c_int32)]
 
 
 class _LayerArgs(C.Structure):
@@ -60,9 +61,13 @@ class _LayerArgs(C.Structure):
                 ("xi_out", C.c_void_p), ("status", C.c_void_p), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p),
                 ("trace_events", C.POINTER(C.c_void_p)), ("seq_rows", C.c_int32), ("aux_stream", C.c_void_p),
-                ("map_event", C.c_void_p)]
+                ("map_event", C.c_void_p), ("fork_event", C.c_void_p), ("join_event", C.c_void_p),
+                ("n_text_ranges", C.c_int32), ("bidirectional", C.c_int32),
+                ("text_ranges", C.POINTER(C.c_int32)),
+                ("lse_out", C.c_void_p), ("lse_out_batch_stride", C.c_int64), ("lse_out_head_stride", C.c_int64)]
 
 
+MAX_TEXT_RANGES = 8
 TRACE_EVENTS = 6
 TRACE_NAMES = ("window_build", "xi", "fd_best_partner", "select_map", "merge_hidden")
 
@@ -140,7 +145,8 @@ class Plan:
     def __init__(self, batch: int, hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
                  n_layers: int, tiles: Sequence[Tuple[int, int]], layers: Sequence[int],
                  windows: Sequence[int], keep: Sequence[float], max_text: int,
-                 dtype: int = BF16, xi_mode: int = XI_ATTN_FULL, engine: int = ENGINE_AUTO):
+                 dtype: int = BF16, xi_mode: int = XI_ATTN_FULL, engine: int = ENGINE_AUTO,
+                 ragged_input: bool = False):
         lib = library()
         n_stages = len(layers)
         self._tiles = (_Tile * len(tiles))(*[_Tile(int(r), int(c)) for r, c in tiles])
@@ -149,7 +155,7 @@ class Plan:
         self._keep = (C.c_double * n_stages)(*[float(v) for v in keep])
         cfg = _Config(C.sizeof(_Config), batch, hidden, n_q_heads, n_kv_heads, head_dim, n_layers,
                       len(tiles), self._tiles, n_stages, self._layers, self._windows, self._keep,
-                      max_text, dtype, xi_mode, engine)
+                      max_text, dtype, xi_mode, engine, int(ragged_input))
         handle = C.c_void_p()
         _check(lib.lightkv_plan(C.byref(cfg), C.byref(handle)), "lightkv_plan")
         self.handle = handle
@@ -217,7 +223,8 @@ def _stream_handle(stream) -> int:
 def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin: int,
                 n_text_after: int = 0, text_begin: int = 0, text_end: Optional[int] = None,
                 q=None, k=None, lse=None, xi=None, n_vis=None, pos=None, stream=None,
-                trace_events=None, aux_stream=None, map_event=None) -> _LayerArgs:
+                trace_events=None, aux_stream=None, map_event=None, fork_event=None, join_event=None,
+                text_ranges=None, bidirectional: bool = False, lse_out=None) -> _LayerArgs:
     a = _LayerArgs()
     a.struct_size = C.sizeof(_LayerArgs)
     a.stage, a.vis_begin, a.n_text_after = stage, vis_begin, n_text_after
@@ -238,7 +245,23 @@ def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin:
     a.workspace, a.workspace_bytes = out.workspace_ptr(), out.info.workspace_bytes
     a.stream = _stream_handle(stream)
     if aux_stream is not None:
+        # the library creates no events: the fork / join pair is the caller's (kept with the stage's buffers here)
+        import torch
         a.aux_stream = aux_stream.cuda_stream
+        if fork_event is None or join_event is None:
+            if not hasattr(out, "fork_join"):
+                out.fork_join = (torch.cuda.Event(), torch.cuda.Event())
+                for e in out.fork_join:
+                    e.record()            # torch creates the CUDA event lazily; the C ABI needs a live handle
+            fork_event, join_event = out.fork_join
+        a.fork_event, a.join_event = fork_event.cuda_event, join_event.cuda_event
+    if text_ranges is not None:       # [(begin, end), ...] instead of the single range text_begin / text_end
+        flat = [int(v) for r in text_ranges for v in r]
+        a._ranges = (C.c_int32 * len(flat))(*flat)          # kept alive by the struct object
+        a.text_ranges, a.n_text_ranges = a._ranges, len(flat) // 2
+    a.bidirectional = int(bool(bidirectional))
+    if lse_out is not None:
+        a.lse_out, a.lse_out_batch_stride, a.lse_out_head_stride = lse_out.data_ptr(), lse_out.stride(0), lse_out.stride(1)
     if map_event is not None:         # a torch.cuda.Event that has been recorded once (torch creates it lazily)
         a.map_event = map_event.cuda_event
     if trace_events is not None:      # TRACE_EVENTS torch.cuda.Event objects (enable_timing=True), already created
@@ -250,7 +273,8 @@ def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin:
 def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, **kw) -> None:
     """lightkv_compress_layer.  hidden [B,N,d]; keywords: vis_begin, n_text_after, text_begin, text_end,
     q [B,H,N,dh], k [B,H_kv,N,dh] (any strides with a contiguous last dimension), lse [B,H,N] fp32,
-    xi [B,cap_in] fp32, n_vis [B] int32, pos [B,cap_in] int32, stream, trace_events, aux_stream, map_event."""
+    xi [B,cap_in] fp32, n_vis [B] int32, pos [B,cap_in] int32, stream, trace_events, aux_stream, map_event,
+    fork_event / join_event, text_ranges [(begin, end), ...], bidirectional, lse_out [B,H,N] fp32."""
     a = _layer_args(plan, stage, hidden, out, **kw)
     _check(library().lightkv_compress_layer(plan.handle, C.byref(a)), "lightkv_compress_layer")
 

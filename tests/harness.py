@@ -35,27 +35,45 @@ def prepare_stage(wl, stage, pos=None, dtype="bf16", samples=None, repair=True, 
     return inp
 
 
-def oracle_stage(wl, stage, inp, xi_mode="attn", n_text_after=0, text_range=None):
+def oracle_stage(wl, stage, inp, xi_mode="attn", n_text_after=0, text_range=None, text_ranges=None, causal=True):
     tb, te = (0, inp["vis_begin"]) if text_range is None else text_range
     q = inp.get("q") if xi_mode in ("attn", "lse") else None
     k = inp.get("k") if xi_mode in ("attn", "lse") else None
     xi = inp.get("xi") if xi_mode == "given" else None
     return O.compress_layer(inp["hidden"], q, k, inp["pos"], inp["n_vis"], inp["vis_begin"], wl.tiles,
                             wl.windows[stage], wl.keep[stage], text_begin=tb, text_end=te, xi=xi,
-                            n_text_after=n_text_after)
+                            n_text_after=n_text_after, causal=causal, text_ranges=text_ranges)
 
 
-def oracle_lse(inp, n_heads, n_kv):
-    """Row log-sum-exp of the scaled causal logits, [B, H, N] (what a fused attention would hand over)."""
-    import scipy.special
-    q, k = inp["q"].astype(np.float64), inp["k"].astype(np.float64)
+def oracle_lse(inp, n_heads, n_kv, causal=True, n_text_after=0, samples=None):
+    """Row log-sum-exp of the scaled logits of the vision rows, [B, H, N] (what a fused attention would hand
+    over; rows outside the vision block stay 0).  Sample b's keys are its own vis_begin + n_vis[b] + n_text_after rows."""
+    q, k = inp["q"], inp["k"]
     b, h, n, dh = q.shape
+    vb = inp["vis_begin"]
     out = np.zeros((b, h, n))
-    mask = np.tril(np.ones((n, n), dtype=bool))
-    for bi in range(b):
+    for bi in (range(b) if samples is None else samples):
+        nv = int(inp["n_vis"][bi])
+        n_seq = vb + nv + n_text_after
         for hi in range(h):
-            logit = q[bi, hi] @ k[bi, hi // (n_heads // n_kv)].T / np.sqrt(dh)
-            out[bi, hi] = scipy.special.logsumexp(np.where(mask, logit, -np.inf), axis=1)
+            out[bi, hi, vb:vb + nv] = O.row_logsumexp(q[bi, hi, :n_seq], k[bi, hi // (n_heads // n_kv), :n_seq],
+                                                     vb, nv, causal)
+    return out
+
+
+def torch_lse(q, k, group):
+    """The same row log-sum-exp (causal) computed with plain torch ops on the device in fp32, for every row: an
+    INPUT of the lse mode at sizes where the float64 oracle would take minutes (the oracle side of the
+    comparison never uses it: it derives xi from Q and K alone)."""
+    import torch
+    b, h, n, dh = q.shape
+    out = torch.empty((b, h, n), dtype=torch.float32, device=q.device)
+    mask = torch.ones((n, n), dtype=torch.bool, device=q.device).tril_()
+    for i in range(b):
+        kk = k[i].float().repeat_interleave(group, dim=0)
+        for h0 in range(0, h, 8):
+            logits = torch.matmul(q[i, h0:h0 + 8].float(), kk[h0:h0 + 8].transpose(1, 2)) / dh ** 0.5
+            out[i, h0:h0 + 8] = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1)
     return out
 
 
@@ -67,18 +85,18 @@ def to_device(arr, dtype, device="cuda"):
     return t.to(device)
 
 
-def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_text=None):
+def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_text=None, ragged=False):
     import paper_2605_00789_b200 as L
     xm = {"attn": L.XI_ATTN_FULL, "lse": L.XI_ATTN_LSE, "given": L.XI_GIVEN, "uniform": L.XI_UNIFORM}[xi_mode]
     return L.Plan(batch or wl.batch, wl.hidden, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_layers,
                   wl.tiles, wl.layers, wl.windows, wl.keep, max_text if max_text is not None else wl.n_text + 64,
                   dtype=L.BF16 if dtype == "bf16" else L.FP32, xi_mode=xm,
-                  engine=L.ENGINE_AUTO if engine == "auto" else L.ENGINE_SIMT)
+                  engine=L.ENGINE_AUTO if engine == "auto" else L.ENGINE_SIMT, ragged_input=ragged)
 
 
 def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0, text_range=None,
               lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None, aux_stream=None,
-              kv_layout="bhnd", kv_stream=None):
+              kv_layout="bhnd", kv_stream=None, text_ranges=None, bidirectional=False, want_lse=False):
     """Run lightkv_compress_layer (or `layer_fn`, a binding function with the same signature) +
     lightkv_compact_kv on the device; returns numpy outputs."""
     import torch
@@ -101,7 +119,20 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
     if xi_mode in ("attn", "lse"):
         kw["q"], kw["k"] = to_device(inp["q"], dtype, device), to_device(inp["k"], dtype, device)
     if xi_mode == "lse":
-        kw["lse"] = torch.from_numpy(lse.astype(np.float32)).to(device)
+        if isinstance(lse, str):          # "torch": computed on the device with plain torch ops
+            kw["lse"] = torch_lse(kw["q"], kw["k"], inp["q"].shape[1] // inp["k"].shape[1])
+        elif isinstance(lse, torch.Tensor):   # already on the device (e.g. the lse_out of an earlier call)
+            kw["lse"] = lse
+        else:
+            kw["lse"] = torch.from_numpy(lse.astype(np.float32)).to(device)
+    if text_ranges is not None:
+        kw["text_ranges"] = text_ranges
+    if bidirectional:
+        kw["bidirectional"] = True
+    lse_out = None
+    if want_lse:
+        lse_out = torch.full((bsz, inp["q"].shape[1], n_seq), float("nan"), dtype=torch.float32, device=device)
+        kw["lse_out"] = lse_out
     cap_pad = info.cap_in - inp["pos"].shape[1]
     assert cap_pad >= 0
     pos = np.pad(inp["pos"], ((0, 0), (0, cap_pad)), constant_values=-1)
@@ -165,6 +196,9 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
     for name in ("n_vis_out", "pos_out", "dst", "weight", "grp_off", "grp_src", "xi_out", "status"):
         res[name] = getattr(out, name).cpu().numpy()
     res["hidden_out"] = out.hidden_out.float().cpu().numpy()
+    if lse_out is not None:
+        res["lse_out"] = lse_out.cpu().numpy()
+        res["lse_out_dev"] = lse_out
     return res
 
 
@@ -227,27 +261,49 @@ def compare_stage(wl, stage, inp, ref, gpu, dtype="bf16", kv_mode="merge", n_tex
     return stats
 
 
+def check_lse_out(inp, gpu, n_heads, n_kv, samples, causal=True, n_text_after=0, atol=2e-3):
+    """lse_out of the vision rows against the oracle's row log-sum-exp (natural log); rows outside the vision
+    block must not have been written (they still hold the NaN fill)."""
+    vb = inp["vis_begin"]
+    want = oracle_lse(inp, n_heads, n_kv, causal, n_text_after, samples=samples)
+    for b in samples:
+        nv = int(inp["n_vis"][b])
+        got = gpu["lse_out"][b]
+        np.testing.assert_allclose(got[:, vb:vb + nv], want[b][:, vb:vb + nv], rtol=0, atol=atol)
+        assert np.isnan(got[:, :vb]).all() and np.isnan(got[:, vb + nv:]).all()
+
+
 def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge", paged=0, samples=None,
-                 stages=None, oracle_samples=None, aux_stream=None, kv_layout="bhnd", kv_stream=None):
-    """All stages of a workload, chained through the surviving positions; returns per-stage stats."""
+                 stages=None, oracle_samples=None, aux_stream=None, kv_layout="bhnd", kv_stream=None,
+                 lse_source="oracle", ragged=False, first_pos=None, text_ranges=None, bidirectional=False,
+                 want_lse=False, expect_status=0):
+    """All stages of a workload, chained through the surviving positions; returns per-stage stats.
+    first_pos: per-sample positions entering stage 0 (a subset of the grid); ragged: plan built for subsets."""
     bsz = wl.batch if samples is None else len(samples)
-    plan = make_plan(wl, dtype, xi_mode, engine, batch=bsz)
-    pos = None
+    plan = make_plan(wl, dtype, xi_mode, engine, batch=bsz, ragged=ragged)
+    pos = first_pos
     all_stats = []
     for stage in (range(wl.n_stages) if stages is None else stages):
         inp = prepare_stage(wl, stage, pos, dtype, samples=samples)
         if xi_mode == "given":
             rng = np.random.default_rng(stage)
             inp["xi"] = rng.uniform(0.05, 3.0, size=inp["pos"].shape).astype(np.float32)
-        lse = oracle_lse(inp, wl.n_q_heads, wl.n_kv_heads) if xi_mode == "lse" else None
+        lse = None
+        if xi_mode == "lse":
+            lse = "torch" if lse_source == "torch" else oracle_lse(inp, wl.n_q_heads, wl.n_kv_heads,
+                                                                   causal=not bidirectional)
         gpu = gpu_stage(plan, wl, stage, inp, dtype, xi_mode, lse=lse, kv_mode=kv_mode, paged=paged,
-                        aux_stream=aux_stream, kv_layout=kv_layout, kv_stream=kv_stream)
+                        aux_stream=aux_stream, kv_layout=kv_layout, kv_stream=kv_stream, text_ranges=text_ranges,
+                        bidirectional=bidirectional, want_lse=want_lse)
         osamp = list(range(bsz)) if oracle_samples is None else oracle_samples
         sub = {key: (val[osamp] if isinstance(val, np.ndarray) and val.shape[:1] == (bsz,) else val)
                for key, val in inp.items()}
-        ref = oracle_stage(wl, stage, sub, xi_mode)
-        stats = compare_stage(wl, stage, inp, ref, gpu, dtype, kv_mode, samples=osamp)
+        ref = oracle_stage(wl, stage, sub, xi_mode, text_ranges=text_ranges, causal=not bidirectional)
+        stats = compare_stage(wl, stage, inp, ref, gpu, dtype, kv_mode, samples=osamp, expect_status=expect_status)
+        if want_lse:
+            check_lse_out(inp, gpu, wl.n_q_heads, wl.n_kv_heads, osamp, causal=not bidirectional)
         stats["n_out"] = [int(v) for v in gpu["n_vis_out"]]
+        stats["info"] = plan.stage_info(stage)
         all_stats.append(stats)
         # chain on the device result (equal to the oracle's on the compared samples)
         pos = [gpu["pos_out"][b, :int(gpu["n_vis_out"][b])] for b in range(bsz)]

@@ -25,7 +25,7 @@ def test_every_declared_symbol_is_exported(L):
     lib = L.library()
     for name in declared:
         assert getattr(lib, name) is not None
-    assert L.version() == 100
+    assert L.version() == 200
     assert L.status_string(0) == "ok" and "workspace" in L.status_string(-3)
 
 
@@ -37,9 +37,9 @@ def test_struct_layouts_match_the_header(L, tmp_path):
 #include <stddef.h>
 #include "lightkv.h"
 int main(void) {
-  printf("%zu %zu\\n", sizeof(lightkv_config_t), offsetof(lightkv_config_t, engine));
-  printf("%zu %zu\\n", sizeof(lightkv_stage_info_t), offsetof(lightkv_stage_info_t, workspace_bytes));
-  printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, map_event));
+  printf("%zu %zu\\n", sizeof(lightkv_config_t), offsetof(lightkv_config_t, ragged_input));
+  printf("%zu %zu\\n", sizeof(lightkv_stage_info_t), offsetof(lightkv_stage_info_t, reserved));
+  printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, lse_out_head_stride));
   printf("%zu %zu\\n", sizeof(lightkv_kv_args_t), offsetof(lightkv_kv_args_t, stream));
   return 0;
 }
@@ -48,9 +48,9 @@ int main(void) {
     subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
     rows = [tuple(int(v) for v in line.split()) for line in subprocess.check_output([str(exe)]).decode().splitlines()]
     k = L.lightkv
-    got = [(C.sizeof(k._Config), k._Config.engine.offset),
-           (C.sizeof(k._StageInfo), k._StageInfo.workspace_bytes.offset),
-           (C.sizeof(k._LayerArgs), k._LayerArgs.map_event.offset),
+    got = [(C.sizeof(k._Config), k._Config.ragged_input.offset),
+           (C.sizeof(k._StageInfo), k._StageInfo.reserved.offset),
+           (C.sizeof(k._LayerArgs), k._LayerArgs.lse_out_head_stride.offset),
            (C.sizeof(k._KvArgs), k._KvArgs.stream.offset)]
     assert got == rows
 
@@ -86,6 +86,7 @@ def test_plan_counts_and_retention(L):
     dict(batch=0), dict(hidden=65), dict(head_dim=12), dict(n_q_heads=3), dict(keep=[0.4, 0.5]),
     dict(keep=[0.5, 1.5]), dict(windows=[7, 1]), dict(windows=[0, 1]), dict(layers=[4, 2]),
     dict(layers=[2, 9]), dict(tiles=[(0, 6)]), dict(dtype=7), dict(xi_mode=9), dict(engine=5),
+    dict(ragged_input=2),
 ])
 def test_plan_rejects_bad_configs(L, kw):
     with pytest.raises(L.LightKVError, match="invalid argument"):
@@ -97,6 +98,68 @@ def test_plan_unsupported(L):
         _plan(L, tiles=[(6, 6)] * 33)
     with pytest.raises(L.LightKVError, match="unsupported"):
         _plan(L, tiles=[(64, 64)], windows=[64, 1])
+    # a window may hold at most 65535 tokens (16-bit counters of the window build): 256 x 256 is one too many
+    _plan(L, tiles=[(255, 257)], windows=[1, 1])
+    with pytest.raises(L.LightKVError, match="unsupported"):
+        _plan(L, tiles=[(256, 256)], windows=[1, 1])
+    _plan(L, tiles=[(510, 514)], windows=[2], layers=[2], keep=[0.5])        # cells of 255 x 257
+    with pytest.raises(L.LightKVError, match="unsupported"):
+        _plan(L, tiles=[(510, 514)], windows=[2, 1])                           # one window at the second stage
+
+
+def test_ragged_input_plans_hold_for_any_subset_of_the_grid(L):
+    """With ragged_input the capacities are bounds over every subset of positions: (cap_in + n_windows) / 2 A
+    nodes and ceil(keep cap_in) + n_windows survivors; a full-grid plan keeps the exact counts."""
+    kw = dict(tiles=[(24, 24)], layers=[12, 18, 24], windows=[6, 4, 2], keep=[0.5] * 3, n_layers=32, hidden=4096,
+              n_q_heads=32, n_kv_heads=32, head_dim=128, batch=1, max_text=64)
+    exact = [L.Plan(**kw).stage_info(s) for s in range(3)]
+    assert [(i.cap_in, i.cap_out, i.counts_exact) for i in exact[:2]] == [(576, 288, 1), (288, 144, 1)]
+    ragged = [L.Plan(ragged_input=True, **kw).stage_info(s) for s in range(3)]
+    assert [(i.cap_in, i.cap_out, i.counts_exact) for i in ragged] == \
+        [(576, 288 + 36, 0), (324, 162 + 16, 0), (178, 89 + 4, 0)]
+    assert all(r.workspace_bytes >= e.workspace_bytes for r, e in zip(ragged, exact))
+
+
+def test_prompt_ranges_and_stream_events_are_checked_on_the_host(L):
+    p = _plan(L)
+    lib = L.library()
+    a = L.lightkv._LayerArgs()
+    a.struct_size = C.sizeof(a)
+    a.vis_begin = 12
+    for f in ("hidden", "n_vis_out", "pos_out", "dst", "weight", "grp_off", "grp_src", "workspace", "q", "k"):
+        setattr(a, f, 0x1000)
+    a.hidden_out = 0x2000
+    a.hidden_row_stride = a.hidden_out_row_stride = 64
+    a.hidden_batch_stride = a.hidden_out_batch_stride = 64 * 64
+    a.q_row_stride = a.k_row_stride = 16
+    a.workspace_bytes = 1 << 30
+
+    def ranges(*pairs):
+        flat = [v for pr in pairs for v in pr]
+        a._keep = (C.c_int32 * len(flat))(*flat)
+        a.text_ranges, a.n_text_ranges = a._keep, len(pairs)
+        return lib.lightkv_compress_layer(p.handle, C.byref(a))
+
+    a.n_text_ranges = 9
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # more ranges than the library takes
+    a.n_text_ranges = 2
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # ranges announced, none given
+    assert ranges((4, 8), (6, 10)) == -1                                     # overlapping
+    assert ranges((6, 10), (0, 4)) == -1                                     # not ascending
+    assert ranges((0, 4), (8, 13)) == -1                                     # reaches into the vision block
+    assert ranges((5, 3)) == -1                                              # end before begin
+    a.n_text_ranges = 0
+    a.bidirectional = 2
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1
+    a.bidirectional = 0
+    a.aux_stream = 0x10
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # second stream without fork / join events
+    a.fork_event = 0x20
+    assert lib.lightkv_compress_layer(p.handle, C.byref(a)) == -1            # ... with only one of them
+    a.aux_stream, a.fork_event = None, None
+    given = _plan(L, xi_mode=L.XI_GIVEN)
+    a.xi, a.lse_out = 0x1000, 0x3000
+    assert lib.lightkv_compress_layer(given.handle, C.byref(a)) == -1        # lse_out needs ATTN_FULL
 
 
 def test_calls_reject_bad_arguments_before_any_launch(L):

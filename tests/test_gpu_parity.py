@@ -174,6 +174,150 @@ def test_run_to_run_bit_repeatability():
         np.testing.assert_array_equal(a[key], b[key])
 
 
+# ---- prompt ranges, rows without the causal mask, the row log-sum-exp as an output ---------------------------
+
+@pytest.mark.parametrize("engine", ["simt", "auto"])
+def test_prompt_ranges_bidirectional_rows_and_lse_out(engine):
+    wl = S.workload("small")                                   # 19 text rows, head_dim 128 (tcgen05 with "auto")
+    H.run_schedule(wl, engine=engine, stages=[0], text_ranges=[(1, 4), (7, 8), (10, 19)], want_lse=True)
+    H.run_schedule(wl, engine=engine, stages=[0, 1], bidirectional=True, want_lse=True)
+    H.run_schedule(wl, engine=engine, stages=[0], bidirectional=True, xi_mode="lse", text_ranges=[(0, 3), (9, 19)])
+
+
+def test_prompt_ranges_over_several_key_tiles():
+    # 200 prompt rows = four 64-key tiles; J = three ranges with holes, cut by tile borders
+    wl = dataclasses.replace(S.workload("cfg0"), n_text=200, hidden=256)
+    ranges = [(3, 50), (60, 70), (100, 190)]
+    H.run_schedule(wl, text_ranges=ranges, want_lse=True)
+    H.run_schedule(wl, text_ranges=ranges, xi_mode="lse")
+    H.run_schedule(wl, text_ranges=ranges, bidirectional=True, want_lse=True)
+
+
+def test_bidirectional_rows_with_text_behind_the_vision_block():
+    # [15 text | vision | 4 text], no causal mask: the rows behind the vision block are keys too (not in J)
+    wl = S.workload("small")
+    plan = H.make_plan(wl)
+    inp = H.prepare_stage(wl, 0)
+    vb, after = wl.n_text - 4, 4
+    for key in ("hidden", "q", "k", "v"):
+        a = inp[key]
+        axis = 1 if key == "hidden" else 2
+        a = np.concatenate([np.take(a, range(0, vb), axis), np.take(a, range(wl.n_text, a.shape[axis]), axis),
+                            np.take(a, range(vb, wl.n_text), axis)], axis)
+        inp[key] = np.ascontiguousarray(a)
+    inp["vis_begin"] = vb
+    gpu = H.gpu_stage(plan, wl, 0, inp, n_text_after=after, text_range=(2, 12), bidirectional=True, want_lse=True)
+    ref = H.oracle_stage(wl, 0, inp, n_text_after=after, text_range=(2, 12), causal=False)
+    H.compare_stage(wl, 0, inp, ref, gpu, n_text_after=after)
+    H.check_lse_out(inp, gpu, wl.n_q_heads, wl.n_kv_heads, range(wl.batch), causal=False, n_text_after=after)
+
+
+@pytest.mark.parametrize("name", ["small", "cfg1"])
+def test_the_librarys_own_row_lse_feeds_the_lse_mode(name):
+    """ATTN_FULL hands out the row log-sum-exp it saw (lse_out); given back as the input of ATTN_LSE, only the
+    prompt keys are visited and xi, the merge map and the merged rows agree with ATTN_FULL and the oracle."""
+    wl = S.workload(name)
+    full, lse_plan = H.make_plan(wl), H.make_plan(wl, xi_mode="lse")
+    inp = H.prepare_stage(wl, 0)
+    a = H.gpu_stage(full, wl, 0, inp, want_lse=True)
+    b = H.gpu_stage(lse_plan, wl, 0, inp, xi_mode="lse", lse=a["lse_out_dev"])
+    ref = H.oracle_stage(wl, 0, inp)
+    H.compare_stage(wl, 0, inp, ref, a)
+    H.compare_stage(wl, 0, inp, ref, b)
+    H.check_lse_out(inp, a, wl.n_q_heads, wl.n_kv_heads, range(wl.batch))
+    for key in ("dst", "grp_src", "grp_off", "pos_out"):
+        np.testing.assert_array_equal(a[key], b[key])
+    nv = int(inp["n_vis"][0])
+    np.testing.assert_allclose(a["xi_out"][:, :nv], b["xi_out"][:, :nv], rtol=2e-3)
+
+
+# ---- persistent CTAs that take more than one work item ---------------------------------------------------------
+
+def _sm_count():
+    import torch
+    return torch.cuda.get_device_properties(0).multi_processor_count
+
+
+@pytest.mark.parametrize("head_dim", [64, 128])
+def test_lse_mode_persistent_ctas_walk_several_items(head_dim):
+    # 4 samples x 8 heads x 16 query tiles = 512 work items for at most 3 CTAs per SM: every CTA of the xi kernel
+    # takes a second item (its barriers and rings run on across items); 130 prompt rows span three key tiles
+    wl = S.Workload(name="lsewalk", config_id=130, batch=4, tiles=((64, 32),), n_text=130, hidden=64, n_q_heads=8,
+                    n_kv_heads=4, head_dim=head_dim, n_layers=16, layers=(3,), windows=(4,), keep=(0.5,))
+    assert 16 * wl.n_q_heads * wl.batch > 3 * _sm_count()
+    H.run_schedule(wl, xi_mode="lse")
+    H.run_schedule(wl, xi_mode="lse", text_ranges=[(2, 60), (70, 129)])
+
+
+def test_cfg2_lse_mode_full_size_sampled():
+    # the benchmark shape in ATTN_LSE mode (5888 work items walked by 3 CTAs per SM), bench.py's streams; the
+    # log-sum-exp input comes from plain torch ops, the oracle derives xi from Q and K alone
+    stats = H.run_schedule(S.workload("cfg2"), xi_mode="lse", lse_source="torch", oracle_samples=[0, 5],
+                           **_bench_streams())
+    assert [s["n_out"] for s in stats] == [[1440] * 8, [720] * 8, [360] * 8]
+
+
+@pytest.mark.parametrize("hidden,ragged", [(64, False), (72, True)])
+def test_fd_persistent_ctas_take_several_tiles(hidden, ragged):
+    # 48 samples x 36 windows of 16 tokens: eight tiles per sample, 384 tiles for the 2 x SMs persistent CTAs of
+    # the tensor-core FD kernel, so CTAs loop over tiles (ring phases and the accumulator barrier run on); the
+    # ragged variant gives every sample its own subset of the grid under a plan built for subsets
+    wl = S.Workload(name="fdmulti", config_id=131, batch=48, tiles=((24, 24),), n_text=4, hidden=hidden,
+                    n_q_heads=2, n_kv_heads=1, head_dim=64, n_layers=16, layers=(3,), windows=(6,), keep=(0.5,))
+    first = None
+    if ragged:
+        rng = np.random.default_rng(77)
+        full = np.arange(wl.n_vis, dtype=np.int32)
+        first = [np.sort(rng.choice(full, int(rng.integers(500, 577)), replace=False)).astype(np.int32)
+                 for _ in range(wl.batch)]
+    stats = H.run_schedule(wl, xi_mode="uniform", oracle_samples=[0, 17, 47], ragged=ragged, first_pos=first)
+    info = stats[0]["info"]
+    assert info.uses_tensor_cores == 1 and info.fd_tiles * wl.batch > 2 * _sm_count()
+
+
+# ---- subsets of the grid: capacities ---------------------------------------------------------------------------
+
+def _near_full_subset():
+    """576-token grid, windows 6 / 4 / 2 (not nested): a sample that misses 8 positions reaches the second stage
+    with 146 A nodes, two more than the full grid's 144 (found with the oracle, seed fixed)."""
+    wl = dataclasses.replace(S.workload("cfg1r"), batch=2, hidden=64, n_q_heads=2, n_kv_heads=2, head_dim=64, n_text=8)
+    rng = np.random.default_rng(9000)
+    full = np.arange(576, dtype=np.int32)
+    n_missing = int(rng.integers(1, 12))
+    subset = np.sort(rng.choice(full, 576 - n_missing, replace=False)).astype(np.int32)
+    return wl, [subset, full]
+
+
+def test_near_full_subset_through_two_stages_under_a_ragged_plan():
+    wl, first = _near_full_subset()
+    stats = H.run_schedule(wl, stages=[0, 1], ragged=True, first_pos=first)
+    assert stats[1]["info"].cap_a >= 146 and stats[1]["info"].counts_exact == 0
+
+
+def test_subset_given_to_a_full_grid_plan_raises_the_count_bit():
+    """The same subset under a plan built for full grids: at the second stage it has more A nodes than the plan
+    holds.  The sample then passes through unmerged (cut at cap_out), the COUNT bit is raised, nothing is written
+    out of a row, and the full-grid sample beside it still matches the oracle."""
+    wl, first = _near_full_subset()
+    plan = H.make_plan(wl, batch=2)
+    inp0 = H.prepare_stage(wl, 0, first)
+    g0 = H.gpu_stage(plan, wl, 0, inp0)
+    H.compare_stage(wl, 0, inp0, H.oracle_stage(wl, 0, inp0), g0)           # stage 0 holds any subset
+    pos1 = [g0["pos_out"][b, :int(g0["n_vis_out"][b])] for b in range(2)]
+    info = plan.stage_info(1)
+    assert info.cap_a == 144 and info.cap_out == 144
+    inp1 = H.prepare_stage(wl, 1, pos1)
+    g1 = H.gpu_stage(plan, wl, 1, inp1)
+    assert int(g1["status"][0]) == 8
+    sub = {k: (v[[1]] if isinstance(v, np.ndarray) and v.shape[:1] == (2,) else v) for k, v in inp1.items()}
+    H.compare_stage(wl, 1, inp1, H.oracle_stage(wl, 1, sub), g1, samples=[1], expect_status=8)
+    vb = inp1["vis_begin"]
+    assert int(g1["n_vis_out"][0]) == info.cap_out
+    np.testing.assert_array_equal(g1["pos_out"][0, :144], pos1[0][:144])
+    np.testing.assert_array_equal(g1["hidden_out"][0, vb:vb + 144], inp1["hidden"][0, vb:vb + 144])
+    plan.close()
+
+
 # ---- seeded random geometries ---------------------------------------------------------------------
 
 def _random_workload(seed):

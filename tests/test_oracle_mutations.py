@@ -113,24 +113,20 @@ def _select_farthest_partner(fd, r):
     return m
 
 
-def _xi_mean_over_heads(q, k, vis_begin, n_vis, text_begin, text_end):
-    return O_xi_from_attention(q, k, vis_begin, n_vis, text_begin, text_end) / q.shape[0]
+def _xi_mean_over_heads(q, k, vis_begin, n_vis, text_begin, text_end, causal=True, text_ranges=None):
+    return O_xi_from_attention(q, k, vis_begin, n_vis, text_begin, text_end, causal, text_ranges) / q.shape[0]
 
 
-def _xi_prompt_range_shifted(q, k, vis_begin, n_vis, text_begin, text_end):
-    return O_xi_from_attention(q, k, vis_begin, n_vis, text_begin + 1, text_end)
+def _xi_prompt_range_shifted(q, k, vis_begin, n_vis, text_begin, text_end, causal=True, text_ranges=None):
+    return O_xi_from_attention(q, k, vis_begin, n_vis, text_begin + 1, text_end, causal, text_ranges)
 
 
-def _attention_without_causal_mask(q, k, vis_begin, n_vis):
-    q, k = np.asarray(q, dtype=F64), np.asarray(k, dtype=F64)
-    logits = (q[vis_begin:vis_begin + n_vis] @ k.T) / math.sqrt(k.shape[1])
-    logits = logits - logits.max(axis=1, keepdims=True)
-    e = np.exp(logits)
-    return e / e.sum(axis=1, keepdims=True)
+def _attention_without_causal_mask(q, k, vis_begin, n_vis, causal=True):
+    return O_attention_rows(q, k, vis_begin, n_vis, False)
 
 
-def _attention_without_scale(q, k, vis_begin, n_vis):
-    return O_attention_rows(np.asarray(q, dtype=F64) * math.sqrt(np.asarray(k).shape[1]), k, vis_begin, n_vis)
+def _attention_without_scale(q, k, vis_begin, n_vis, causal=True):
+    return O_attention_rows(np.asarray(q, dtype=F64) * math.sqrt(np.asarray(k).shape[1]), k, vis_begin, n_vis, causal)
 
 
 def _message_passing_plain_mean(xa, xb, xi_a, xi_b, m):
@@ -140,6 +136,39 @@ def _message_passing_plain_mean(xa, xb, xi_a, xi_b, m):
 def _message_passing_transposed_weights(xa, xb, xi_a, xi_b, m):
     # the A-side weights applied in reversed order (a transposed / mis-indexed operand)
     return O_message_passing(xa, xb, np.asarray(xi_a, dtype=F64)[::-1].copy(), xi_b, m)
+
+
+def _message_passing_without_the_zero_sum_fallback(xa, xb, xi_a, xi_b, m):
+    # the vanishing-denominator branch dropped: the division runs on whatever the sums are
+    xa, xb = np.asarray(xa, dtype=F64), np.asarray(xb, dtype=F64)
+    xi_a, xi_b = np.asarray(xi_a, dtype=F64), np.asarray(xi_b, dtype=F64)
+    mt = m.T.astype(F64)
+    den = xi_b + mt @ xi_a
+    with np.errstate(all="ignore"):
+        num = xb * xi_b[:, None] + mt @ (xa * xi_a[:, None])
+        return num / den[:, None], (m.astype(F64) @ (1.0 / den)) * xi_a, xi_b / den
+
+
+def _message_passing_fallback_hits_every_group(xa, xb, xi_a, xi_b, m):
+    # one vanishing sum switches ALL groups to the plain mean
+    xi_a, xi_b = np.asarray(xi_a, dtype=F64), np.asarray(xi_b, dtype=F64)
+    den = xi_b + m.T.astype(F64) @ xi_a
+    if (den < 1e-30).any():
+        return O_message_passing(xa, xb, np.ones_like(xi_a), np.ones_like(xi_b), m)
+    return O_message_passing(xa, xb, xi_a, xi_b, m)
+
+
+def _row_logsumexp_without_the_scale(q, k, vis_begin, n_vis, causal=True):
+    return O_row_logsumexp(np.asarray(q, dtype=F64) * math.sqrt(np.asarray(k).shape[1]), k, vis_begin, n_vis, causal)
+
+
+def _xi_first_range_only(q, k, vis_begin, n_vis, text_begin, text_end, causal=True, text_ranges=None):
+    return O_xi_from_attention(q, k, vis_begin, n_vis, text_begin, text_end, causal,
+                               None if text_ranges is None else list(text_ranges)[:1])
+
+
+def _scaled_logits_always_causal(q, k, vis_begin, n_vis, causal=True):
+    return O_scaled_logits(q, k, vis_begin, n_vis, True)
 
 
 def _window_of_swapped_axes(pos, tiles, w):
@@ -157,6 +186,7 @@ def _compact_kv_ignores_the_weights(kv, vis_begin, n_vis, dst, weight, survivor,
 O_feature_divergence, O_removal_count, O_xi_from_attention = O.feature_divergence, O.removal_count, O.xi_from_attention
 O_attention_rows, O_message_passing, O_window_of = O.attention_rows, O.message_passing, O.window_of
 O_retention, O_compact_kv = O.retention, O.compact_kv
+O_row_logsumexp, O_scaled_logits = O.row_logsumexp, O.scaled_logits
 
 MUTATIONS = [
     ("feature_divergence", _fd_wrong_sign),
@@ -173,6 +203,11 @@ MUTATIONS = [
     ("attention_rows", _attention_without_scale),
     ("message_passing", _message_passing_plain_mean),
     ("message_passing", _message_passing_transposed_weights),
+    ("message_passing", _message_passing_without_the_zero_sum_fallback),
+    ("message_passing", _message_passing_fallback_hits_every_group),
+    ("row_logsumexp", _row_logsumexp_without_the_scale),
+    ("xi_from_attention", _xi_first_range_only),
+    ("scaled_logits", _scaled_logits_always_causal),
     ("window_of", _window_of_swapped_axes),
     ("retention", _retention_counts_the_compression_layer_as_compressed),
     ("compact_kv", _compact_kv_ignores_the_weights),

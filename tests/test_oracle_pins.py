@@ -207,6 +207,60 @@ def test_xi_equals_exp_of_logit_minus_logsumexp():
     np.testing.assert_allclose(xi, want, rtol=1e-12)
 
 
+def test_xi_without_the_causal_mask_is_the_equation_as_printed():
+    # causal=False: every query sees all N keys.  Library softmax row by row; zero queries give H |J| / N.
+    rng = np.random.default_rng(15)
+    n_heads, n_kv, n_text, n_vis, dh = 4, 2, 6, 7, 8
+    n_seq = n_text + n_vis
+    q, k = _rand_qk(rng, n_heads, n_kv, n_seq, dh)
+    xi = O.xi_from_attention(q, k, n_text, n_vis, 1, 5, causal=False)
+    want = np.zeros(n_vis)
+    for h in range(n_heads):
+        for t in range(n_vis):
+            p = scipy.special.softmax(k[h // 2] @ q[h, n_text + t] / math.sqrt(dh))
+            want[t] += p[1:5].sum()
+    np.testing.assert_allclose(xi, want, rtol=1e-12)
+    xi0 = O.xi_from_attention(np.zeros_like(q), k, n_text, n_vis, 0, n_text, causal=False)
+    np.testing.assert_allclose(xi0, n_heads * n_text / n_seq, rtol=1e-13)
+    a = O.attention_rows(q[0], k[0], n_text, n_vis, causal=False)
+    np.testing.assert_allclose(a.sum(axis=1), 1.0, rtol=1e-13)
+    assert (a[0, n_text + 1:] > 0).all()                   # keys behind the query are visible
+    # the last query sees every key either way
+    np.testing.assert_allclose(O.attention_rows(q[0], k[0], n_text, n_vis)[-1], a[-1], rtol=1e-13)
+
+
+def test_xi_over_several_prompt_ranges_is_the_sum_over_the_ranges():
+    rng = np.random.default_rng(16)
+    n_heads, n_text, n_vis, dh = 3, 12, 5, 8
+    q, k = _rand_qk(rng, n_heads, n_heads, n_text + n_vis, dh)
+    parts = [O.xi_from_attention(q, k, n_text, n_vis, lo, hi) for lo, hi in ((1, 3), (5, 6), (8, 12))]
+    both = O.xi_from_attention(q, k, n_text, n_vis, 0, 0, text_ranges=[(1, 3), (5, 6), (8, 12)])
+    np.testing.assert_allclose(both, sum(parts), rtol=1e-13)
+    whole = O.xi_from_attention(q, k, n_text, n_vis, 0, n_text)
+    gaps = O.xi_from_attention(q, k, n_text, n_vis, 0, 0, text_ranges=[(0, 1), (3, 5), (6, 8)])
+    np.testing.assert_allclose(both + gaps, whole, rtol=1e-13)
+
+
+def test_row_logsumexp_against_the_library():
+    rng = np.random.default_rng(17)
+    n_text, n_vis, dh = 4, 6, 16
+    q, k = rng.standard_normal((n_text + n_vis, dh)), rng.standard_normal((n_text + n_vis, dh))
+    logit = q @ k.T / math.sqrt(dh)
+    got = O.row_logsumexp(q, k, n_text, n_vis)
+    want = [scipy.special.logsumexp(logit[n_text + t, :n_text + t + 1]) for t in range(n_vis)]
+    np.testing.assert_allclose(got, want, rtol=1e-13)
+    got = O.row_logsumexp(q, k, n_text, n_vis, causal=False)
+    np.testing.assert_allclose(got, scipy.special.logsumexp(logit[n_text:], axis=1), rtol=1e-13)
+    # shifting every logit of a row by c shifts the result by c: scale a query so that its logits are huge
+    big = q.copy()
+    big[n_text] *= 400.0
+    assert np.isfinite(O.row_logsumexp(big, k, n_text, n_vis)).all()
+    # and it is the normaliser of the attention rows
+    a = O.attention_rows(q, k, n_text, n_vis)
+    np.testing.assert_allclose(np.exp(logit[n_text:, :n_text] - O.row_logsumexp(q, k, n_text, n_vis)[:, None]),
+                               a[:, :n_text], rtol=1e-12)
+
+
 # ------------------------------------------------------------- merge (Eq. "message-passing")
 
 def _case(seed, n=36, d=12, tiles=((6, 6),), w=1, keep=0.5):
@@ -260,6 +314,39 @@ def test_uniform_xi_is_the_group_mean_and_xi_scale_is_irrelevant():
     big[a0] = 1e6
     r3 = O.compress_vision(x, pos, big, tiles, w, keep)
     np.testing.assert_allclose(r3["x_out"][r3["dst"][a0]], x[a0], atol=1e-4)
+
+
+def test_vanishing_xi_sum_falls_back_to_the_plain_group_mean():
+    """A group whose xi sum is (numerically) zero cannot be normalised: it takes the plain mean of its members
+    and weights 1 / size; groups with a proper sum beside it are left alone; weights still sum to one."""
+    rng = np.random.default_rng(18)
+    xa, xb = rng.standard_normal((3, 5)), rng.standard_normal((2, 5))
+    m = np.array([[1, 0], [1, 0], [0, 1]])                 # A0, A1 -> B0;  A2 -> B1
+    xi_a, xi_b = np.array([0.0, 0.0, 0.7]), np.array([0.0, 1.3])
+    xb_new, w_a, w_b = O.message_passing(xa, xb, xi_a, xi_b, m)
+    np.testing.assert_allclose(xb_new[0], (xb[0] + xa[0] + xa[1]) / 3.0, rtol=1e-14)
+    np.testing.assert_allclose([w_b[0], w_a[0], w_a[1]], 1.0 / 3.0, rtol=1e-15)
+    np.testing.assert_allclose(xb_new[1], (1.3 * xb[1] + 0.7 * xa[2]) / 2.0, rtol=1e-14)
+    np.testing.assert_allclose([w_b[1], w_a[2]], [0.65, 0.35], rtol=1e-14)
+    assert w_b[0] + w_a[0] + w_a[1] == pytest.approx(1.0, abs=1e-15) and w_b[1] + w_a[2] == pytest.approx(1.0, abs=1e-15)
+    # an untouched B node with xi = 0 keeps its own row (a group of one)
+    xb_new, w_a, w_b = O.message_passing(xa, xb, np.array([0.5, 0.5, 0.5]), np.array([0.0, 0.0]),
+                                         np.array([[1, 0], [0, 0], [0, 0]]))
+    np.testing.assert_allclose(xb_new[0], xa[0], rtol=1e-14)          # all of the group's mass sits on A0
+    np.testing.assert_array_equal(xb_new[1], xb[1])
+    assert w_b[1] == 1.0
+    # through the whole step: xi = 0 everywhere gives the same result as uniform xi
+    x, pos, _, tiles, w, keep = _case(19)
+    r0 = O.compress_vision(x, pos, np.zeros(len(x)), tiles, w, keep)
+    r1 = O.compress_vision(x, pos, np.ones(len(x)), tiles, w, keep)
+    np.testing.assert_allclose(r0["x_out"], r1["x_out"], rtol=1e-14)
+    np.testing.assert_allclose(r0["weight"], r1["weight"], rtol=1e-15)
+    # tiny but representable sums are still normalised by xi
+    tiny = np.full(len(x), 1e-20)
+    tiny[0] = 3e-20
+    r2 = O.compress_vision(x, pos, tiny, tiles, w, keep)
+    r3 = O.compress_vision(x, pos, tiny * 1e20, tiles, w, keep)
+    np.testing.assert_allclose(r2["x_out"], r3["x_out"], rtol=1e-12)
 
 
 def test_direction_is_a_into_b_and_position_of_group_is_b():

@@ -53,9 +53,23 @@ def test_builtin_workspace_matches_caller_workspace_on_two_calls_in_a_row():
     first = H.prepare_stage(wl, 0, repair=False)
     second = H.prepare_stage(wl, 0, ragged, repair=False)
 
+    # Free device memory is read right around the entry point itself (every buffer it is given exists by then).
+    # The first call on a device loads the library's kernels and its fixed scratch array; from then on a call
+    # must leave the amount of free memory where it found it.
+    moved = []
+
+    def watched(*args, **kw):
+        torch.cuda.synchronize()
+        before = torch.cuda.mem_get_info()[0]
+        L.compress_layer_builtin_ws(*args, **kw)
+        torch.cuda.synchronize()
+        moved.append(before - torch.cuda.mem_get_info()[0])
+
+    H.gpu_stage(plan, wl, 0, first, layer_fn=L.compress_layer_builtin_ws)      # loads kernels and the array
     for inp in (first, second):                   # two calls in a row on the shared array
-        got = H.gpu_stage(plan, wl, 0, inp, layer_fn=L.compress_layer_builtin_ws)
+        got = H.gpu_stage(plan, wl, 0, inp, layer_fn=watched)
         want = H.gpu_stage(plan, wl, 0, inp)
         assert int(want["status"][0]) == 0
         _same(got, want, [int(n) for n in inp["n_vis"]])
+    assert moved == [0, 0], f"free device memory moved across the calls: {moved}"
     plan.close()
