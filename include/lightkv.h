@@ -75,6 +75,17 @@ extern "C" {
 #define LIGHTKV_ENGINE_AUTO 0    /* tcgen05 tensor-core kernels for bf16 where the shape allows */
 #define LIGHTKV_ENGINE_SIMT 1    /* fp32 FMA kernels                                            */
 
+/* pair score of Step 2 (appendix "Influence of similarity metrics"); the method uses the first */
+#define LIGHTKV_FD_COSINE 0      /* FD = 1 - cosine, Eq. "similarity"     */
+#define LIGHTKV_FD_L2SQ   1      /* squared Euclidean distance            */
+#define LIGHTKV_FD_L2     2      /* Euclidean distance                    */
+
+/* direction of the messages (paragraph "Token message passing": "the reverse direction can be defined
+ * analogously") */
+#define LIGHTKV_DIR_A2B 0        /* A nodes (1st, 3rd, ... token of a window) are merged into B nodes: the method */
+#define LIGHTKV_DIR_B2A 1        /* the sets swap roles: B nodes are merged into their best A node; a window of
+                                    n tokens can then lose at most floor(n / 2) of them                           */
+
 typedef struct lightkv_plan lightkv_plan_t;
 
 typedef struct { int32_t rows, cols; } lightkv_tile_t;   /* grid of one image tile / video frame */
@@ -106,6 +117,8 @@ typedef struct {
                                          cap_a = (cap_in + n_windows) / 2, cap_out = ceil(keep cap_in) +
                                          n_windows.  A subset given to a plan built with 0 is still safe:
                                          a sample that overflows a capacity raises LIGHTKV_STATUS_COUNT. */
+  int32_t  divergence;             /* LIGHTKV_FD_* */
+  int32_t  direction;              /* LIGHTKV_DIR_* */
 } lightkv_config_t;
 
 typedef struct {

@@ -140,6 +140,24 @@ def feature_divergence(xa: np.ndarray, xb: np.ndarray) -> np.ndarray:
     return 1.0 - cos
 
 
+def divergence(xa: np.ndarray, xb: np.ndarray, metric: str = "cosine") -> np.ndarray:
+    """Pair scores for all (a, b), [|A|, |B|]; lower = more alike.
+    "cosine": FD of Eq. "similarity" (the method).  "l2sq" / "l2": squared and plain
+    Euclidean distance, the two alternatives of appendix "Influence of similarity
+    metrics" (they rank pairs alike; both are kept because both are named)."""
+    if metric == "cosine":
+        return feature_divergence(xa, xb)
+    xa = np.asarray(xa, dtype=F64)
+    xb = np.asarray(xb, dtype=F64)
+    diff = xa[:, None, :] - xb[None, :, :]
+    sq = (diff * diff).sum(axis=2)
+    if metric == "l2sq":
+        return sq
+    if metric == "l2":
+        return np.sqrt(sq)
+    raise ValueError(metric)
+
+
 def removal_count(n_window: int, keep: float) -> int:
     """Tokens removed from a window of n tokens: floor(rho * n) with rho = 1 - keep,
     at most |A| = ceil(n / 2) (a step cannot remove more than half: "Limitations"),
@@ -212,8 +230,15 @@ def message_passing(xa: np.ndarray, xb: np.ndarray, xi_a: np.ndarray, xi_b: np.n
 # --------------------------------------------------------------------------
 
 def compress_vision(x: np.ndarray, pos: np.ndarray, xi: np.ndarray,
-                    tiles: Sequence[Tuple[int, int]], w: int, keep: float) -> Dict[str, np.ndarray]:
+                    tiles: Sequence[Tuple[int, int]], w: int, keep: float,
+                    metric: str = "cosine", direction: str = "a2b") -> Dict[str, np.ndarray]:
     """x [n, d], pos [n] (original flat positions, any storage order), xi [n].
+
+    metric: pair score of Step 2 (see divergence).  direction: "a2b" passes messages
+    from X_A to X_B as the method does; "b2a" is the reverse direction that paragraph
+    "Token message passing" says can be defined analogously: the two sets swap
+    roles, so B nodes are merged into their best A node and at most |B| = floor(n / 2)
+    tokens of a window disappear.
 
     Returns
       x_out [n_out, d]  survivors (all B nodes, updated, and the unconnected A
@@ -243,9 +268,13 @@ def compress_vision(x: np.ndarray, pos: np.ndarray, xi: np.ndarray,
         ia, ib = bipartition(members)
         if len(ib) == 0:
             continue
-        fd = feature_divergence(x[ia], x[ib])
+        if direction == "b2a":
+            ia, ib = ib, ia                             # sources are the B nodes, destinations the A nodes
+        elif direction != "a2b":
+            raise ValueError(direction)
+        fd = divergence(x[ia], x[ib], metric)
         fd_best[ia] = fd.min(axis=1)
-        r = removal_count(len(members), keep)
+        r = min(removal_count(len(members), keep), len(ia))
         m = select_edges(fd, r)
         xb_new, w_a, w_b = message_passing(x[ia], x[ib], xi[ia], xi[ib], m)
         touched = m.sum(axis=0) > 0
@@ -267,12 +296,13 @@ def compress_vision(x: np.ndarray, pos: np.ndarray, xi: np.ndarray,
 
 
 def compress_sequence(hidden: np.ndarray, vis_begin: int, n_vis: int, pos: np.ndarray,
-                      xi: np.ndarray, tiles: Sequence[Tuple[int, int]], w: int, keep: float
-                      ) -> Dict[str, np.ndarray]:
+                      xi: np.ndarray, tiles: Sequence[Tuple[int, int]], w: int, keep: float,
+                      metric: str = "cosine", direction: str = "a2b") -> Dict[str, np.ndarray]:
     """Whole sequence of one sample: text rows are copied, the vision block
     [vis_begin, vis_begin + n_vis) is compressed in place of itself."""
     hidden = np.asarray(hidden, dtype=F64)
-    res = compress_vision(hidden[vis_begin:vis_begin + n_vis], pos[:n_vis], xi[:n_vis], tiles, w, keep)
+    res = compress_vision(hidden[vis_begin:vis_begin + n_vis], pos[:n_vis], xi[:n_vis], tiles, w, keep,
+                          metric, direction)
     res["hidden_out"] = np.concatenate(
         [hidden[:vis_begin], res["x_out"], hidden[vis_begin + n_vis:]], axis=0)
     return res
@@ -356,8 +386,8 @@ def compress_layer(hidden: np.ndarray, q: Optional[np.ndarray], k: Optional[np.n
                    tiles: Sequence[Tuple[int, int]], w: int, keep: float,
                    text_begin: int = 0, text_end: Optional[int] = None,
                    xi: Optional[np.ndarray] = None, n_text_after: int = 0, causal: bool = True,
-                   text_ranges: Optional[Sequence[Tuple[int, int]]] = None
-                   ) -> List[Dict[str, np.ndarray]]:
+                   text_ranges: Optional[Sequence[Tuple[int, int]]] = None,
+                   metric: str = "cosine", direction: str = "a2b") -> List[Dict[str, np.ndarray]]:
     """One compression stage on a batch (samples are independent).
     hidden [B, N, d]; q [B, H, N, dh]; k [B, H_kv, N, dh]; pos [B, cap]; n_vis [B].
     Sample b's sequence is [text (vis_begin rows) | n_vis[b] vision rows | n_text_after rows];
@@ -375,7 +405,8 @@ def compress_layer(hidden: np.ndarray, q: Optional[np.ndarray], k: Optional[np.n
                                      causal, text_ranges)
         else:
             xi_b = np.ones(nv, dtype=F64)
-        res = compress_sequence(hidden[b][:n_seq], vis_begin, nv, pos[b][:nv], xi_b, tiles, w, keep)
+        res = compress_sequence(hidden[b][:n_seq], vis_begin, nv, pos[b][:nv], xi_b, tiles, w, keep,
+                                metric, direction)
         res["xi"] = xi_b
         out.append(res)
     return out

@@ -5,6 +5,6 @@ Importing the package does not load the library; the first call does and fails l
 shared object has not been built (see __graft_entry__.build)."""
 from .lightkv import (  # noqa: F401
     BF16, FP32, XI_GIVEN, XI_ATTN_FULL, XI_ATTN_LSE, XI_UNIFORM, KV_MERGE, KV_GATHER,
-    ENGINE_AUTO, ENGINE_SIMT, LightKVError, Plan, StageBuffers, compress_layer, compress_layer_builtin_ws, BUILTIN_WS_BYTES, compact_kv,
+    ENGINE_AUTO, ENGINE_SIMT, FD_COSINE, FD_L2SQ, FD_L2, DIR_A2B, DIR_B2A, MAX_TEXT_RANGES, LightKVError, Plan, StageBuffers, compress_layer, compress_layer_builtin_ws, BUILTIN_WS_BYTES, compact_kv,
     library, library_path, status_string, version, TRACE_EVENTS, TRACE_NAMES,
 )

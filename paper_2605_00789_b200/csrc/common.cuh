@@ -18,6 +18,7 @@ struct Geometry {
   int n_tiles;
   int w;                               // windows per axis, per tile
   int n_windows;                       // n_tiles * w * w
+  int src_par;                         // parity of the local rank of the source nodes (0: A -> B, 1: B -> A)
   int tile_off[kMaxTiles + 1];         // first flat position of each tile
   int rows[kMaxTiles];
   int cols[kMaxTiles];
@@ -81,8 +82,10 @@ struct TextSet {
 };
 
 // Tokens removed from a window of n tokens when a fraction `keep` must remain:
-// floor((1 - keep) n) evaluated as n - ceil(keep n - 1e-9), at most ceil(n / 2), none without a B node.
-__host__ __device__ inline int removal_count(int n, double keep) {
+// floor((1 - keep) n) evaluated as n - ceil(keep n - 1e-9), at most the number of source nodes (the tokens
+// of local rank parity `src_par`: ceil(n / 2) A nodes, or floor(n / 2) B nodes in the reverse direction), none
+// from a window of one token.
+__host__ __device__ inline int removal_count(int n, double keep, int src_par = 0) {
   if (n < 2) return 0;
 #ifdef __CUDA_ARCH__
   double t = __dadd_rn(__dmul_rn(keep, (double)n), -1e-9);
@@ -91,7 +94,7 @@ __host__ __device__ inline int removal_count(int n, double keep) {
   double t = prod - 1e-9;
 #endif
   int r = n - (int)ceil(t);
-  int na = (n + 1) >> 1;
+  int na = (n + 1 - src_par) >> 1;
   return r < 0 ? 0 : (r > na ? na : r);
 }
 

@@ -33,7 +33,7 @@ inline cudaError_t launch_kernel(void (*kernel)(P...), dim3 grid, dim3 block, si
 
 struct LayerLaunch {
   int batch, hidden, n_q_heads, n_kv_heads, head_dim;
-  int dtype, xi_mode;
+  int dtype, xi_mode, divergence;
   double keep;
   int fd_tiles;                      // estimate of FdTiling::n_tiles per sample (launch shape of the tensor-core FD kernel)
   Geometry geo;

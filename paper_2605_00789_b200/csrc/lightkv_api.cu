@@ -119,6 +119,8 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
   if (c->xi_mode < LIGHTKV_XI_GIVEN || c->xi_mode > LIGHTKV_XI_UNIFORM) return LIGHTKV_ERR_INVALID_ARG;
   if (c->engine != LIGHTKV_ENGINE_AUTO && c->engine != LIGHTKV_ENGINE_SIMT) return LIGHTKV_ERR_INVALID_ARG;
   if (c->ragged_input != 0 && c->ragged_input != 1) return LIGHTKV_ERR_INVALID_ARG;
+  if (c->divergence < LIGHTKV_FD_COSINE || c->divergence > LIGHTKV_FD_L2) return LIGHTKV_ERR_INVALID_ARG;
+  if (c->direction != LIGHTKV_DIR_A2B && c->direction != LIGHTKV_DIR_B2A) return LIGHTKV_ERR_INVALID_ARG;
   if (c->n_tiles > kMaxTiles) return LIGHTKV_ERR_UNSUPPORTED;
   if (c->head_dim > 256) return LIGHTKV_ERR_UNSUPPORTED;
 
@@ -149,6 +151,7 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
         (s > 0 && sp.layer <= c->layers[s - 1])) { delete p; return LIGHTKV_ERR_INVALID_ARG; }
     Geometry& g = sp.geo;
     g.n_tiles = c->n_tiles; g.w = sp.w; g.n_windows = c->n_tiles * sp.w * sp.w;
+    g.src_par = c->direction == LIGHTKV_DIR_B2A ? 1 : 0;
     g.tile_off[0] = 0;
     for (int t = 0; t < c->n_tiles; ++t) {
       if (sp.w > p->tiles[t].rows || sp.w > p->tiles[t].cols) { delete p; return LIGHTKV_ERR_INVALID_ARG; }
@@ -172,10 +175,11 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
       int cap_a = 0, cap_b = 0, max_a = 0;
       bool still = true;
       for (const auto& m : members) {
-        const int n = (int)m.size(), na = (n + 1) / 2, r = removal_count(n, sp.keep);
-        cap_a += na; cap_b += n / 2;
-        max_a = std::max(max_a, na);
-        if (r == na && n >= 2) { for (int l = 1; l < n; l += 2) next.push_back(m[l]); }
+        // sources: the tokens of local rank parity src_par; the others are the destinations and always survive
+        const int n = (int)m.size(), na = (n + 1 - g.src_par) / 2, r = removal_count(n, sp.keep, g.src_par);
+        cap_a += na; cap_b += n - na;
+        max_a = std::max(max_a, std::max(na, n - na));
+        if (r == na && n >= 2) { for (int l = 1 - g.src_par; l < n; l += 2) next.push_back(m[l]); }
         else if (r == 0) { next.insert(next.end(), m.begin(), m.end()); }
         else still = false;
       }
@@ -189,9 +193,9 @@ int lightkv_plan(const lightkv_config_t* c, lightkv_plan_t** out) {
         exact = false;
       }
     }
-    if (!sp.exact) {
-      sp.cap_a = (sp.cap_in + sp.n_windows) / 2;
-      sp.cap_b = sp.cap_in / 2;
+    if (!sp.exact) {      // sum over windows of ceil(n_w / 2) resp. floor(n_w / 2), whichever set is the source
+      sp.cap_a = g.src_par ? sp.cap_in / 2 : (sp.cap_in + sp.n_windows) / 2;
+      sp.cap_b = g.src_par ? (sp.cap_in + sp.n_windows) / 2 : sp.cap_in / 2;
     }
     if (!sp.exact) {  // counts depend on the data: a window holds at most the tokens of its grid cell
                       // (balanced cells: ceil(rows/w) x ceil(cols/w))
@@ -302,7 +306,8 @@ int lightkv_compress_layer(const lightkv_plan_t* p, const lightkv_layer_args_t* 
 
   LayerLaunch L;
   L.batch = c.batch; L.hidden = c.hidden; L.n_q_heads = c.n_q_heads; L.n_kv_heads = c.n_kv_heads;
-  L.head_dim = c.head_dim; L.dtype = c.dtype; L.xi_mode = c.xi_mode; L.keep = s.keep; L.geo = s.geo;
+  L.head_dim = c.head_dim; L.dtype = c.dtype; L.xi_mode = c.xi_mode; L.divergence = c.divergence;
+  L.keep = s.keep; L.geo = s.geo;
   L.fd_tiles = s.fd_tiles;
   L.ws = bind_workspace(s, a->workspace); L.text = text; L.a = a; L.stream = static_cast<cudaStream_t>(a->stream);
 

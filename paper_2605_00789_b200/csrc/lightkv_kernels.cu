@@ -15,7 +15,9 @@ __device__ inline void set_status(uint32_t* status, uint32_t bit) {
 // Window build ("Window partitioning", Step 1).  One CTA per sample.
 // Every token gets its window id from its original grid position; tokens of a window are ranked in
 // storage order (positions ascend with storage, so this is position order).  Rank l even -> set A
-// (the paper's 1st, 3rd, ... token), odd -> set B.  A and B nodes are listed window by window.
+// (the paper's 1st, 3rd, ... token), odd -> set B.  The SOURCE nodes (the ones that may be merged away: set A,
+// or set B in the reverse direction, g.src_par = 1) go to the a_* lists, the destinations to b_tok, window by
+// window.
 // Stable ranking without sorting: each warp owns a contiguous segment of the tokens and a private row
 // of per-window counters; an exclusive prefix over the 32 rows gives every warp its starting rank.
 // =====================================================================================================
@@ -83,7 +85,7 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
     const int chunk = (nW + 31) / 32;
     const int lo = min(nW, lane * chunk), hi = min(nW, lo + chunk);
     int s = 0, sa = 0;
-    for (int w = lo; w < hi; ++w) { s += wsum[w]; sa += (wsum[w] + 1) >> 1; }
+    for (int w = lo; w < hi; ++w) { s += wsum[w]; sa += (wsum[w] + 1 - g.src_par) >> 1; }
     int xs = s, xa = sa;
     for (int o = 1; o < 32; o <<= 1) {
       const int t = __shfl_up_sync(0xffffffffu, xs, o), ta = __shfl_up_sync(0xffffffffu, xa, o);
@@ -93,7 +95,7 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
     for (int w = lo; w < hi; ++w) {
       const int c = wsum[w];
       wsum[w] = xs; asum[w] = xa;
-      xs += c; xa += (c + 1) >> 1;
+      xs += c; xa += (c + 1 - g.src_par) >> 1;
     }
     if (lane == 31) { wsum[nW] = xs; asum[nW] = xa; }
   }
@@ -123,19 +125,21 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
       mb = __reduce_max_sync(0xffffffffu, max_ab[1][lane]);
       if (lane == 0) {
         FdTiling t;
-        if (ma <= kFdTile) {
-          // as few windows per tile as still gives the batch about kFdTargetTiles tiles, at most 128 A entries
+        const int mm = max(ma, mb);                      // either side of a window (the destinations outnumber the
+                                                         // sources by one per odd window in the reverse direction)
+        if (mm <= kFdTile) {
+          // as few windows per tile as still gives the batch about kFdTargetTiles tiles, at most 128 entries a side
           const int want = (nW * (int)gridDim.x + kFdTargetTiles - 1) / kFdTargetTiles;
-          t.wpt = ma > 0 ? max(1, min(min(kFdTile / ma, nW), want)) : nW;
+          t.wpt = mm > 0 ? max(1, min(min(kFdTile / mm, nW), want)) : nW;
           t.blocks_a = 1; t.blocks_b = 1;
-          const int rows = t.wpt * ma;
+          const int rows = t.wpt * mm;
           t.passes = rows <= 32 ? 1 : (rows <= 64 ? 2 : 4);
         } else {
           t.wpt = 1;
           t.blocks_a = (ma + kFdTile - 1) / kFdTile; t.blocks_b = (mb + kFdTile - 1) / kFdTile;
           t.passes = 4;
         }
-        t.n_tiles = (mb > 0 && !over) ? ((nW + t.wpt - 1) / t.wpt) * t.blocks_a * t.blocks_b : 0;
+        t.n_tiles = (ma > 0 && mb > 0 && !over) ? ((nW + t.wpt - 1) / t.wpt) * t.blocks_a * t.blocks_b : 0;
         t.pad[0] = t.pad[1] = t.pad[2] = 0;
         ws.fd_tiling[b] = t;
       }
@@ -156,7 +160,7 @@ window_build_kernel(Geometry g, const int* __restrict__ pos_all, const int* __re
       __syncwarp(amask);
       const int l = before + __popc(peers & ((1u << lane) - 1u));
       tok_l[i] = l;
-      if (l & 1) {
+      if ((l & 1) != g.src_par) {
         const int e = (wsum[w] - asum[w]) + (l >> 1);
         if (e < ws.cap_b) b_tok[e] = i;
       } else {
@@ -202,7 +206,7 @@ __device__ inline void load4<__nv_bfloat16>(const __nv_bfloat16* p, float (&f)[4
 template <typename T>
 __global__ void __launch_bounds__(256)
 fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_stride, int vis_begin,
-               int d, Workspace ws) {
+               int d, int metric, Workspace ws) {
   grid_dependency_sync();
   __shared__ float As[FD_TA][FD_KC + 1];
   __shared__ float Bs[FD_TB][FD_KC + 1];
@@ -293,9 +297,14 @@ fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_s
       const int lo = max(a_lo[tid], cb), hi = min(a_hi[tid], cb + nb);
       const float na = sqrtf(a_ss[tid]);
       for (int e = lo; e < hi; ++e) {
-        const float den = na * sqrtf(b_ss[e - cb]);
-        const float cosv = den > 0.f ? Gs[tid][e - cb] / den : 0.f;
-        const float fd = 1.0f - cosv;
+        float fd;
+        if (metric == LIGHTKV_FD_COSINE) {
+          const float den = na * sqrtf(b_ss[e - cb]);
+          fd = 1.0f - (den > 0.f ? Gs[tid][e - cb] / den : 0.f);
+        } else {
+          fd = fmaxf(fmaf(-2.0f, Gs[tid][e - cb], a_ss[tid] + b_ss[e - cb]), 0.f);   // |a|^2 + |b|^2 - 2 <a, b>
+          if (metric == LIGHTKV_FD_L2) fd = sqrtf(fd);
+        }
         if (fd < best_f) { best_f = fd; best_e = e; }
       }
     }
@@ -310,9 +319,9 @@ cudaError_t launch_fd_simt(const LayerLaunch& L) {
   if (L.dtype == LIGHTKV_BF16)
     return launch_kernel(fd_simt_kernel<__nv_bfloat16>, grid, 256, 0, L.stream, 1,
                          static_cast<const __nv_bfloat16*>(L.a->hidden), L.a->hidden_batch_stride,
-                         L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.ws);
+                         L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.divergence, L.ws);
   return launch_kernel(fd_simt_kernel<float>, grid, 256, 0, L.stream, 1, static_cast<const float*>(L.a->hidden),
-                       L.a->hidden_batch_stride, L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.ws);
+                       L.a->hidden_batch_stride, L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.divergence, L.ws);
 }
 
 // =====================================================================================================
@@ -482,7 +491,7 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
 // CTA keeps a contiguous range of the sample's tokens through all phases, phases that read what other
 // threads wrote are separated by cluster barriers, prefix sums cross the cluster through distributed shared
 // memory.
-//   1  xi = fixed-order sum over heads (or given / uniform); every A token (even local rank): r =
+//   1  xi = fixed-order sum over heads (or given / uniform); every source token (local rank parity src_par): r =
 //      removal_count(n_w), selected iff it is among the r entries of its window with the smallest
 //      (FD, index) (rank by counting 32-bit keys; skipped when r = |A|); a selected token takes its best B
 //   2  survivors (all B, unselected A) get consecutive output slots in storage (= position) order: dst,
@@ -494,7 +503,7 @@ cudaError_t launch_xi_simt(const LayerLaunch& L) {
 //   6  weights xi_i / sum over the group, the sum taken in that fixed order
 // =====================================================================================================
 struct SelectArgs {
-  int n_q_heads, xi_mode, cap_out;
+  int n_q_heads, xi_mode, cap_out, src_par;
   double keep;
   const int* n_vis;
   const int* pos;
@@ -628,11 +637,11 @@ __global__ void __launch_bounds__(1024) select_map_kernel(Workspace ws, SelectAr
     if (a.xi_out) a.xi_out[size_t(b) * ws.cap_in + i] = v;
     int p = -1;
     const int l = tok_l[i];
-    if (!(l & 1)) {
+    if ((l & 1) == a.src_par) {                        // a source node
       const int w = tok_win[i];
       const int e_lo = a_off[w], e_hi = a_off[w + 1], e = e_lo + (l >> 1);
       if (e < ws.cap_a) {
-        const int r = removal_count(win_off[w + 1] - win_off[w], a.keep);
+        const int r = removal_count(win_off[w + 1] - win_off[w], a.keep, a.src_par);
         bool sel;
         if (r <= 0) sel = false;
         else if (r >= e_hi - e_lo) sel = true;
@@ -721,6 +730,7 @@ cudaError_t launch_select_map(const LayerLaunch& L) {
   const lightkv_layer_args_t* a = L.a;
   SelectArgs s;
   s.n_q_heads = L.n_q_heads; s.xi_mode = L.xi_mode; s.cap_out = L.ws.cap_out; s.keep = L.keep;
+  s.src_par = L.geo.src_par;
   s.n_vis = a->n_vis; s.pos = a->pos; s.xi_in = a->xi; s.n_vis_out = a->n_vis_out; s.pos_out = a->pos_out;
   s.dst = a->dst; s.weight = a->weight; s.grp_off = a->grp_off; s.grp_src = a->grp_src;
   s.xi_out = a->xi_out; s.status = a->status;

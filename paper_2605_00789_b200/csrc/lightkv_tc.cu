@@ -46,22 +46,45 @@ static bool make_map_bhnd(CUtensorMap* map, const void* base, int width, int row
 }
 
 // ======================================================================================================
-// xi per head on tensor cores (Eq. "attention-factor" over the causal softmax rows of Eq.
-// "attention-matrix").
+// xi per head on tensor cores (Eq. "attention-factor" over the softmax rows of Eq. "attention-matrix").
 //
 // A work item is (tile of 128 vision queries, head, sample); three CTAs share an SM.  Warp 0 streams the Q
 // tile once and the K tiles (64 keys) through a 2-stage ring with TMA; warp 1 issues S = Q K^T (128 x 64 x dh,
 // bf16 -> fp32) into one of two TMEM accumulators; warps 2-5 own one query row per thread (= TMEM lane), pull
-// the 64 logits of the row into registers, release the accumulator, and fold them into a running maximum and
-// two running sums (all visible keys / prompt keys J).  Tiles that straddle the diagonal are masked, and the
-// columns no row of a warp can see are skipped; only tiles that reach into J take the prompt-sum path.
-// Output per head: sum_J / sum_all.  With the caller's row log-sum-exp only the prompt key tiles are visited
-// and the CTAs walk the item list (WALK), so that an item's loads overlap the previous item's arithmetic.
+// the 64 logits of the row into registers, release the accumulator, and add exp(logit - reference) to two
+// sums per row (all visible keys / prompt keys J).  Output per head: sum_J / sum_all.
+//
+// The kernel is bound by the exponentials (one per logit on the special-function unit, 16 per clock per SM,
+// against one MMA per tile), so the softmax arithmetic is kept to three instructions per logit:
+//   * the reference subtracted before the exponential is the row's maximum over the FIRST key tile only
+//     (softmax is invariant to the reference; fp32 holds exp of any later logit up to 88 above it), so the
+//     other tiles need no maximum and no rescaling;
+//   * on tiles that need neither the causal mask nor the prompt mask, every fourth exponential is evaluated
+//     on the FMA pipe instead (range reduction + cubic, relative error 7.5e-5), which takes a quarter of the
+//     load off the special-function unit.
+// A row whose sum left the fp32 range (a later logit more than 88 above the first tile's maximum) is found at
+// the end of the item: the CTA then repeats the item with a running maximum and rescaling, as an ordinary
+// online softmax does, and overwrites its results.  Tiles that straddle the diagonal (or the end of the
+// sample) are masked, and the columns no row of a warp can see are skipped.
+// With the caller's row log-sum-exp (WALK) only the prompt key tiles are visited and the CTAs walk the item
+// list, so that an item's loads overlap the previous item's arithmetic.
 // ======================================================================================================
 __device__ __forceinline__ float ex2(float x) {          // one MUFU op, flush-to-zero
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// 2^x on the FMA and integer pipes: x is clamped to [-126, 128], split into the nearest integer j (magic-number
+// add) and r in [-0.5, 0.5]; 2^r by a minimax cubic; j is added to the exponent field.  x = 128 gives the bit
+// pattern of a non-finite value, which the overflow check at the end of the item sees.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fminf(fmaxf(x, -126.f), 128.f);
+  const float t = x + 12582912.f;                         // 1.5 * 2^23: the integer lands in the low mantissa bits
+  const float r = x - (t - 12582912.f);
+  float p = fmaf(r, 0.0551716685f, 0.2426111251f);
+  p = fmaf(p, r, 0.6932609677f);
+  p = fmaf(p, r, 0.9999280572f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
 
 struct XiTcArgs {
@@ -80,17 +103,20 @@ struct XiTcArgs {
 };
 
 constexpr int XT_STAGES = 2;
-constexpr int XT_KEY_TILE = 64;      // keys per tile (64: three CTAs per SM; 128: two)
+constexpr int XT_KEY_TILE = 64;      // keys per tile: two 64-column accumulators per CTA, three CTAs per SM
 
+// WALK = true <=> the caller supplied the row log-sum-exp (a.lse != nullptr).
 template <int DH, int BK, bool WALK>
-__global__ void __launch_bounds__(192, BK == 64 ? 3 : 2)
+__global__ void __launch_bounds__(192, 3)
 xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, XiTcArgs a) {
   grid_dependency_sync();
+  static_assert(BK == 64, "the prompt mask of a tile is one 64-bit word");
   constexpr int HALVES = DH / 64;
   constexpr uint32_t TILE_BYTES = HALVES * 16384;          // Q tile: 128 rows x DH bf16
   constexpr uint32_t KHALF_BYTES = BK * 128;               // BK key rows x 64 columns
   constexpr uint32_t KT_BYTES = HALVES * KHALF_BYTES;      // K tile: BK rows x DH bf16
   constexpr int NC = BK / 32;                              // 32-column chunks of a tile
+  constexpr int N_PASS = WALK ? 1 : 2;                     // second pass: the item again, with a running maximum
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* q_s = base;
@@ -102,8 +128,10 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   uint64_t* s_full = k_empty + XT_STAGES;      // [2]
   uint64_t* s_empty = s_full + 2;              // [2]
   uint64_t* q_empty = s_empty + 2;             // every MMA that reads the Q tile has completed
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_empty + 1);
+  uint64_t* verdict = q_empty + 1;             // the four softmax warps have checked their sums of the first pass
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(verdict + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* redo = const_cast<int*>(abort_flag) + 1;            // some row's sum left the fp32 range
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Work items: (query tile, head, sample), the query tiles of one head next to each other (they share its K
@@ -113,7 +141,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   const int n_items = WALK ? a.n_qt * a.n_q_heads * a.batch : 0;
   // key tiles to visit: all tiles up to the last query's own key, or, when the caller supplies the row
   // log-sum-exp, only the tiles that hold prompt keys (J lies before the vision block, so it is visible)
-  const int kt_lo = a.lse ? a.text.begin / BK : 0;
+  const int kt_lo = WALK ? a.text.begin / BK : 0;
   const int nkt_lse = a.text.end > a.text.begin ? (a.text.end - 1) / BK + 1 - kt_lo : 0;
   struct Item { int h, b, t0, nq, s_first, nkt, n_seq; };
   auto decode = [&](int item, Item& it) -> bool {
@@ -130,7 +158,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     it.nq = min(128, n - it.t0);
     it.s_first = a.vis_begin + it.t0;
     it.n_seq = a.vis_begin + n + a.n_text_after;
-    it.nkt = a.lse ? nkt_lse : ((a.bidirectional ? it.n_seq : it.s_first + it.nq) - 1) / BK + 1;
+    it.nkt = WALK ? nkt_lse : ((a.bidirectional ? it.n_seq : it.s_first + it.nq) - 1) / BK + 1;
     return true;
   };
   Item it0 = {};
@@ -138,10 +166,12 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    if (WALK) mbar_init(q_empty, 1);
+    mbar_init(q_empty, 1);
+    mbar_init(verdict, 4);
     for (int i = 0; i < XT_STAGES; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4); }
     *abort_flag = 0;
+    *redo = 0;
     fence_barrier_init();
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 2 * BK); tmem_relinquish(); }
@@ -159,19 +189,24 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       for (int item = blockIdx.x; ok && (!WALK || item < n_items); item += gridDim.x) {
         Item it = it0;
         if ((WALK && !decode(item, it)) || it.nkt == 0) { if (WALK) continue; else break; }
-        // the Q tile is free once every MMA of the previous item has completed
-        if (WALK && done > 0 && !mbar_wait(q_empty, (done - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(q_full, TILE_BYTES);
+        for (int pass = 0; ok && pass < N_PASS; ++pass) {
+          if (pass == 1 && (!mbar_wait(verdict, 0, abort_flag) || !*redo)) break;
+          if (pass == 0) {
+            // the Q tile is free once every MMA of the previous item has completed
+            if (WALK && done > 0 && !mbar_wait(q_empty, (done - 1) & 1, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(q_full, TILE_BYTES);
 #pragma unroll
-        for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.s_first, it.h, it.b);
-        const int hk = it.h / a.group;
-        for (int kt = 0; kt < it.nkt; ++kt, ++kf) {
-          const uint32_t s = kf % XT_STAGES;
-          if (!mbar_wait(&k_empty[s], ((kf / XT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(&k_full[s], KT_BYTES);
+            for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.s_first, it.h, it.b);
+          }
+          const int hk = it.h / a.group;
+          for (int kt = 0; kt < it.nkt; ++kt, ++kf) {
+            const uint32_t s = kf % XT_STAGES;
+            if (!mbar_wait(&k_empty[s], ((kf / XT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(&k_full[s], KT_BYTES);
 #pragma unroll
-          for (int hf = 0; hf < HALVES; ++hf)
-            tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, it.b);
+            for (int hf = 0; hf < HALVES; ++hf)
+              tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, it.b);
+          }
         }
         ++done;
         if (!WALK) break;
@@ -186,19 +221,22 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       for (int item = blockIdx.x; ok && (!WALK || item < n_items); item += gridDim.x) {
         Item it = it0;
         if ((WALK && !decode(item, it)) || it.nkt == 0) { if (WALK) continue; else break; }
-        if (!mbar_wait(q_full, done & 1, abort_flag)) break;
-        for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
-          const uint32_t s = kc % XT_STAGES, buf = kc & 1;
-          if (!mbar_wait(&s_empty[buf], ((kc >> 1) & 1) ^ 1, abort_flag) ||
-              !mbar_wait(&k_full[s], (kc / XT_STAGES) & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
+        for (int pass = 0; ok && pass < N_PASS; ++pass) {
+          if (pass == 1 && (!mbar_wait(verdict, 0, abort_flag) || !*redo)) break;
+          if (pass == 0 && !mbar_wait(q_full, done & 1, abort_flag)) { ok = false; break; }
+          for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
+            const uint32_t s = kc % XT_STAGES, buf = kc & 1;
+            if (!mbar_wait(&s_empty[buf], ((kc >> 1) & 1) ^ 1, abort_flag) ||
+                !mbar_wait(&k_full[s], (kc / XT_STAGES) & 1, abort_flag)) { ok = false; break; }
+            tc_fence_after();
 #pragma unroll
-          for (int kk = 0; kk < DH / 16; ++kk) {
-            umma_bf16(tmem_base + buf * BK, smem_desc_sw128(q_addr + (kk >> 2) * 16384 + (kk & 3) * 32),
-                      smem_desc_sw128(k_addr + s * KT_BYTES + (kk >> 2) * KHALF_BYTES + (kk & 3) * 32), idesc, kk > 0);
+            for (int kk = 0; kk < DH / 16; ++kk) {
+              umma_bf16(tmem_base + buf * BK, smem_desc_sw128(q_addr + (kk >> 2) * 16384 + (kk & 3) * 32),
+                        smem_desc_sw128(k_addr + s * KT_BYTES + (kk >> 2) * KHALF_BYTES + (kk & 3) * 32), idesc, kk > 0);
+            }
+            umma_commit(&k_empty[s]);
+            umma_commit(&s_full[buf]);
           }
-          umma_commit(&k_empty[s]);
-          umma_commit(&s_full[buf]);
         }
         if (WALK && ok) umma_commit(q_empty);
         ++done;
@@ -216,120 +254,120 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       Item it = it0;
       if (WALK && !decode(item, it)) continue;
       const int h = it.h, b = it.b, nq = it.nq, s_first = it.s_first;
-      float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
-      for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
-        const uint32_t buf = kc & 1;
-        const int j0 = (kt_lo + kt) * BK;
-        const bool landed = mbar_wait(&s_full[buf], (kc >> 1) & 1, abort_flag);
-        if (!__all_sync(0xffffffffu, landed)) { alive = false; break; }   // the TMEM loads below are warp-wide
-        tc_fence_after();
-        float v[NC][32];
-#pragma unroll
-        for (int c = 0; c < NC; ++c) tmem_ld32(lane_addr + buf * BK + c * 32, v[c]);
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_empty[buf]);
-
-        if (a.lse) {                                      // normaliser known: only the prompt columns count
-          const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
-          const unsigned long long tm = a.text.mask64(j0);     // BK <= 64 columns
-          float st = 0.f;
-#pragma unroll
-          for (int c = 0; c < NC; ++c)
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if ((tm >> (c * 32 + i)) & 1ull) st += ex2(fmaf(v[c][i], sc, -l2));
-          l_txt += st;
-          l_all = 1.f;
-          continue;
+      for (int pass = 0; alive && pass < N_PASS; ++pass) {
+        if (pass == 1) {
+          const bool known = mbar_wait(verdict, 0, abort_flag);
+          if (!__all_sync(0xffffffffu, known)) { alive = false; break; }
+          if (!*redo) break;
         }
-        const bool in_j = j0 < a.text.end && j0 + BK > a.text.begin;   // tile reaches into the prompt set J
-        if (j0 + BK - 1 > (a.bidirectional ? it.n_seq - 1 : s_first)) {
-          // ---- tile straddles the diagonal (or, without the causal mask, the end of the sample): mask.  Columns
-          // beyond the warp's last visible one are skipped in blocks of eight (a warp-uniform test), so most of
-          // the masked half costs no exponentials.
-          const int lim = (a.bidirectional ? it.n_seq - 1 : s_first + r) - j0;   // last visible column of this row (may be negative)
-          const int lim_max = __reduce_max_sync(0xffffffffu, lim);
-          if (lim_max < 0) continue;                      // no row of this warp sees any key of the tile
+        const bool safe = pass == 1;                      // running maximum on every tile
+        float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
+        for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
+          const uint32_t buf = kc & 1;
+          const int j0 = (kt_lo + kt) * BK;
+          const bool landed = mbar_wait(&s_full[buf], (kc >> 1) & 1, abort_flag);
+          if (!__all_sync(0xffffffffu, landed)) { alive = false; break; }   // the TMEM loads below are warp-wide
+          tc_fence_after();
+          float v[NC][32];
 #pragma unroll
-          for (int c = 0; c < NC; ++c)
+          for (int c = 0; c < NC; ++c) tmem_ld32(lane_addr + buf * BK + c * 32, v[c]);
+          tmem_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s_empty[buf]);
+
+          if (WALK) {                                       // normaliser known: only the prompt columns count
+            const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
+            const unsigned long long tm = a.text.mask64(j0);
+            float st = 0.f;
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c * 32 + i > lim) v[c][i] = -INFINITY;
-          if (!in_j) {
-            float mxd[NC];
+            for (int c = 0; c < NC; ++c)
 #pragma unroll
-            for (int c = 0; c < NC; ++c) {
-              mxd[c] = v[c][0];
+              for (int i = 0; i < 32; ++i)
+                if ((tm >> (c * 32 + i)) & 1ull) st += ex2(fmaf(v[c][i], sc, -l2));
+            l_txt += st;
+            l_all = 1.f;
+            continue;
+          }
+          const bool in_j = j0 < a.text.end && j0 + BK > a.text.begin;   // tile reaches into the prompt set J
+          // some row of the tile does not see all of its keys: the diagonal, or the end of the sample
+          const bool edge = j0 + BK - 1 > (a.bidirectional ? it.n_seq - 1 : s_first);
+          int lim_max = BK;                                // columns at least one row of this warp sees
+          if (edge) {
+            const int lim = (a.bidirectional ? it.n_seq - 1 : s_first + r) - j0;   // last visible column of this row
+            lim_max = __reduce_max_sync(0xffffffffu, lim);
+            if (lim_max < 0) continue;                     // no row of this warp sees any key of the tile
 #pragma unroll
-              for (int i = 1; i < 32; ++i) mxd[c] = fmaxf(mxd[c], v[c][i]);
+            for (int c = 0; c < NC; ++c)
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (c * 32 + i > lim) v[c][i] = -INFINITY;
+          }
+          if (kt == 0 || safe) {
+            // reference of the row: maximum of the first tile (every row sees key 0), of every tile when safe
+            float mx[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              mx[j] = v[j / 2][(j & 1) * 16];
+#pragma unroll
+              for (int i = 1; i < 16; ++i) mx[j] = fmaxf(mx[j], v[j / 2][(j & 1) * 16 + i]);
             }
-            float m_new = m_run;                            // finite from the second tile on; tile 0 shows key 0 to every row
+            const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), m_run);
+            const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
+            l_all *= resc;
+            l_txt *= resc;
+            m_run = m_new;
+          }
+          const float ms = m_run * sc;
+          if (!edge && !in_j) {
+            // the bulk of the tiles: every fourth exponential on the FMA pipe
+            float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < NC; ++c) m_new = fmaxf(m_new, mxd[c]);
-            const float ms = m_new * sc;
-            float sa = 0.f;
+            for (int c = 0; c < NC; ++c)
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                const float x = fmaf(v[c][i], sc, -ms);
+                part[(i & 1) + 2 * c] += (i & 3) == 3 ? ex2_fma(x) : ex2(x);
+              }
+            l_all += (part[0] + part[1]) + (part[2] + part[3]);
+          } else {
+            const unsigned long long tm = in_j ? a.text.mask64(j0) : 0ull;
+            float sa = 0.f, st = 0.f;
 #pragma unroll
             for (int c = 0; c < NC; ++c)
 #pragma unroll
               for (int blk = 0; blk < 4; ++blk)
-                if (c * 32 + blk * 8 <= lim_max) {
-                  float part = 0.f;
+                if (c * 32 + blk * 8 <= lim_max) {          // warp-uniform: masked blocks cost no exponentials
+                  float pa = 0.f, pt = 0.f;
 #pragma unroll
-                  for (int i = 0; i < 8; ++i) part += ex2(fmaf(v[c][blk * 8 + i], sc, -ms));
-                  sa += part;
+                  for (int i = 0; i < 8; ++i) {
+                    const float p = ex2(fmaf(v[c][blk * 8 + i], sc, -ms));   // exp2(-inf) = 0 on masked columns
+                    pa += p;
+                    if ((tm >> (c * 32 + blk * 8 + i)) & 1ull) pt += p;
+                  }
+                  sa += pa;
+                  st += pt;
                 }
-            const float resc = ex2((m_run - m_new) * sc);
-            l_all = fmaf(l_all, resc, sa);
-            l_txt *= resc;
-            m_run = m_new;
-            continue;
+            l_all += sa;
+            l_txt += st;
           }
         }
-        float mxc[NC];                                     // one dependency chain per 32-column chunk
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-          mxc[c] = v[c][0];
-#pragma unroll
-          for (int i = 1; i < 32; ++i) mxc[c] = fmaxf(mxc[c], v[c][i]);
+        if (!alive) break;
+        if (!WALK && pass == 0) {
+          // a sum that is not a finite positive number means some logit lay more than 88 above the reference
+          const bool bad = r < nq && !(l_all <= 3.0e38f);
+          const bool any_bad = __any_sync(0xffffffffu, bad);
+          if (lane == 0) {
+            if (any_bad) atomicOr(redo, 1);
+            mbar_arrive(verdict);
+          }
         }
-        float m_new = m_run;
-#pragma unroll
-        for (int c = 0; c < NC; ++c) m_new = fmaxf(m_new, mxc[c]);
-        const float ms = m_new * sc;
-        float sa = 0.f, st = 0.f;
-        if (in_j) {
-          const unsigned long long tm = a.text.mask64(j0);     // BK <= 64 columns
-#pragma unroll
-          for (int c = 0; c < NC; ++c)
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float p = ex2(fmaf(v[c][i], sc, -ms));
-              sa += p;
-              if ((tm >> (c * 32 + i)) & 1ull) st += p;
-            }
-        } else {
-          float part[NC];                                   // independent sums
-#pragma unroll
-          for (int c = 0; c < NC; ++c) part[c] = 0.f;
-#pragma unroll
-          for (int c = 0; c < NC; ++c)
-#pragma unroll
-            for (int i = 0; i < 32; ++i) part[c] += ex2(fmaf(v[c][i], sc, -ms));
-#pragma unroll
-          for (int c = 0; c < NC; ++c) sa += part[c];
+        if (r < nq && !*abort_flag) {
+          a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + it.t0 + r] = WALK ? l_txt : l_txt / l_all;
+          if (!WALK && a.lse_out)
+            a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + s_first + r] =
+                fmaf(m_run, sc, log2f(l_all)) * 0.6931471805599453f;
         }
-        const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
-        l_all = fmaf(l_all, resc, sa);
-        l_txt = fmaf(l_txt, resc, st);
-        m_run = m_new;
-      }
-      if (alive && r < nq && !*abort_flag) {
-        a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + it.t0 + r] = a.lse ? l_txt : l_txt / l_all;
-        if (a.lse_out)
-          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + s_first + r] =
-              fmaf(m_run, sc, log2f(l_all)) * 0.6931471805599453f;
       }
       if (!WALK) break;
     }
@@ -414,9 +452,21 @@ struct FdTcArgs {
   const __nv_bfloat16* x;              // first vision row of sample 0
   int64_t batch_stride, row_stride;    // elements
   int d, batch;
+  int metric;                          // LIGHTKV_FD_*
   Workspace ws;
   uint32_t* status;
 };
+
+// pair score from the inner product g and the norms of the two rows: the norms themselves for FD = 1 - cosine,
+// the squared norms for the Euclidean scores |a|^2 + |b|^2 - 2 g
+__device__ __forceinline__ float pair_score(int metric, float g, float na, float nb) {
+  if (metric == LIGHTKV_FD_COSINE) {
+    const float den = na * nb;
+    return 1.0f - (den > 0.f ? g / den : 0.f);
+  }
+  const float sq = fmaxf(fmaf(-2.0f, g, na + nb), 0.f);
+  return metric == LIGHTKV_FD_L2 ? sqrtf(sq) : sq;
+}
 
 constexpr int FT_LOADERS = 256;
 constexpr int FT_STAGES = 6;
@@ -430,7 +480,7 @@ constexpr size_t FT_SMEM = size_t(FT_RING_BYTES) + 1024 /* alignment */ + 128 /*
 // Second half of the cluster epilogue (kept out of line so that it does not weigh on the registers of the
 // streaming loop): full norms = partial squared sums added in rank order; then CTA `rank` finishes rows
 // [rank * 128 / ks, (rank + 1) * 128 / ks), a warp per row, lanes over the columns of the row's window.
-__device__ __noinline__ void fd_cluster_finish(const int* a_win, unsigned long long* a_key, int ks, int rank, int a0, int a1,
+__device__ __noinline__ void fd_cluster_finish(int metric, const int* a_win, unsigned long long* a_key, int ks, int rank, int a0, int a1,
                                                int b0, int b1,
                                                bool combine, const int* win_off, const int* a_off, uint32_t p0,
                                                const float* a_nrm, const float* b_nrm, float* nrm_a, float* nrm_b,
@@ -441,7 +491,7 @@ __device__ __noinline__ void fd_cluster_finish(const int* a_win, unsigned long l
     const uint32_t src = smem_u32(tid < kFdTile ? a_nrm + i : b_nrm + i);
     float ss = 0.f;
     for (int j = 0; j < ks; ++j) ss += ld_cluster_f32(map_to_cta(src, j));
-    (tid < kFdTile ? nrm_a : nrm_b)[i] = sqrtf(ss);
+    (tid < kFdTile ? nrm_a : nrm_b)[i] = metric == LIGHTKV_FD_COSINE ? sqrtf(ss) : ss;
   }
   named_barrier(1, FT_LOADERS);
   // CTA `rank` finishes rows [rank * 128 / ks, (rank + 1) * 128 / ks): a warp per row, lanes over the
@@ -459,8 +509,7 @@ __device__ __noinline__ void fd_cluster_finish(const int* a_win, unsigned long l
       const uint32_t src = p0 + uint32_t(row * kFdPitch + col) * 4;
       float gsum = 0.f;
       for (int j = 0; j < ks; ++j) gsum += ld_cluster_f32(map_to_cta(src, j));
-      const float den = na * nrm_b[col];
-      const float fd = 1.0f - (den > 0.f ? gsum / den : 0.f);
+      const float fd = pair_score(metric, gsum, na, nrm_b[col]);
       if (fd < best) { best = fd; best_c = col; }
     }
 #pragma unroll
@@ -631,9 +680,8 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         const uint4 v = ld_shared16(sb + t * 4096);
         if (odd) acc_o[t] = sumsq(v, acc_o[t]); else acc_e[t] = sumsq(v, acc_e[t]);
       }
-      fence_proxy_async();                                // cp.async writes -> visible to the tensor core
       __syncwarp();
-      if (lane == 0) mbar_arrive(&full[s_cur]);
+      if (lane == 0) mbar_arrive(&full[s_cur]);           // the MMA warp fences the proxies after its wait
     }
     cp_async_wait<0>();
 
@@ -651,8 +699,9 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         ssb[i] += __shfl_xor_sync(0xffffffffu, ssb[i], o);
       }
       if (c == 0 && i < passes) {                         // a cluster exchanges the squared partial sums
-        a_nrm[g + 32 * i] = ks == 1 ? sqrtf(ssa[i]) : ssa[i];
-        b_nrm[g + 32 * i] = ks == 1 ? sqrtf(ssb[i]) : ssb[i];
+        const bool root = ks == 1 && a.metric == LIGHTKV_FD_COSINE;
+        a_nrm[g + 32 * i] = root ? sqrtf(ssa[i]) : ssa[i];
+        b_nrm[g + 32 * i] = root ? sqrtf(ssb[i]) : ssb[i];
       }
     }
     named_barrier(1, FT_LOADERS);
@@ -697,8 +746,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         for (int i = 0; i < 32; ++i) {
           const int col = c0 + i;
           if (col >= lo && col < hi) {
-            const float den = na * b_nrm[col];
-            const float fd = 1.0f - (den > 0.f ? v[i] / den : 0.f);
+            const float fd = pair_score(a.metric, v[i], na, b_nrm[col]);
             if (fd < best) { best = fd; best_c = col; }
           }
         }
@@ -731,6 +779,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
         const uint32_t FA = done + 2 * k, FB = FA + 1, sA = FA % FT_STAGES, sB = FB % FT_STAGES;
         if (!mbar_wait(&full[sA], (FA / FT_STAGES) & 1, abort_flag)) break;
         if (!mbar_wait(&full[sB], (FB / FT_STAGES) & 1, abort_flag)) break;
+        fence_proxy_async();                              // the loaders' cp.async writes -> visible to the tensor core
         tc_fence_after();
         chunk_mma(ring + sA * FT_STAGE_BYTES, ring + sB * FT_STAGE_BYTES, k == 0);
         umma_commit(&empty[sA]);
@@ -740,6 +789,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       for (int f = 0; f < nf; ++f) {
         const uint32_t F = done + f, s = F % FT_STAGES;
         if (!mbar_wait(&full[s], (F / FT_STAGES) & 1, abort_flag)) break;
+        fence_proxy_async();
         tc_fence_after();
         const uint32_t sa = ring + s * FT_STAGE_BYTES;
         if (passes == 2) {
@@ -759,7 +809,7 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     __syncwarp();
     cluster_sync();                                       // all partial G and squared norms are in shared memory
     if (warp < 8)
-      fd_cluster_finish(a.ws.a_win + size_t(b) * a.ws.cap_a, a.ws.a_key + size_t(b) * a.ws.cap_a, ks, rank, a0, a1, b0, b1,
+      fd_cluster_finish(a.metric, a.ws.a_win + size_t(b) * a.ws.cap_a, a.ws.a_key + size_t(b) * a.ws.cap_a, ks, rank, a0, a1, b0, b1,
                         tl.blocks_b > 1, win_off, a_off, smem_u32(base), a_nrm, b_nrm, red_f,
                         reinterpret_cast<float*>(red_c), abort_flag);
     __syncwarp();
@@ -798,7 +848,7 @@ cudaError_t launch_fd_tc(const LayerLaunch& L) {
   FdTcArgs f;
   f.x = static_cast<const __nv_bfloat16*>(a->hidden) + size_t(a->vis_begin) * a->hidden_row_stride;
   f.batch_stride = a->hidden_batch_stride; f.row_stride = a->hidden_row_stride; f.d = L.hidden; f.batch = L.batch;
-  f.ws = L.ws; f.status = a->status;
+  f.metric = L.divergence; f.ws = L.ws; f.status = a->status;
   // Persistent CTAs, two per SM, no more than the plan expects tiles.  When that estimate leaves SMs idle,
   // clusters of 2, 4 or 8 CTAs split the hidden dimension of every tile.
   const long long bound = std::max<long long>(1, (long long)L.fd_tiles * L.batch);   // an estimate, see the plan

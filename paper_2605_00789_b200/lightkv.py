@@ -13,6 +13,8 @@ BF16, FP32 = 0, 1
 XI_GIVEN, XI_ATTN_FULL, XI_ATTN_LSE, XI_UNIFORM = 0, 1, 2, 3
 KV_MERGE, KV_GATHER = 0, 1
 ENGINE_AUTO, ENGINE_SIMT = 0, 1
+FD_COSINE, FD_L2SQ, FD_L2 = 0, 1, 2
+DIR_A2B, DIR_B2A = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
@@ -33,7 +35,8 @@ class _Config(C.Structure):
                 ("n_stages", C.c_int32), ("layers", C.POINTER(C.c_int32)),
                 ("windows", C.POINTER(C.c_int32)), ("keep", C.POINTER(C.c_double)),
                 ("max_text", C.c_int32), ("dtype", C.c_int32), ("xi_mode", C.c_int32),
-                ("engine", C.c_int32), ("ragged_input", C.c_int32)]
+                ("engine", C.c_int32), ("ragged_input", C.c_int32), ("divergence", C.c_int32),
+                ("direction", C.c_int32)]
 
 
 class _StageInfo(C.Structure):
@@ -146,7 +149,7 @@ class Plan:
                  n_layers: int, tiles: Sequence[Tuple[int, int]], layers: Sequence[int],
                  windows: Sequence[int], keep: Sequence[float], max_text: int,
                  dtype: int = BF16, xi_mode: int = XI_ATTN_FULL, engine: int = ENGINE_AUTO,
-                 ragged_input: bool = False):
+                 ragged_input: bool = False, divergence: int = FD_COSINE, direction: int = DIR_A2B):
         lib = library()
         n_stages = len(layers)
         self._tiles = (_Tile * len(tiles))(*[_Tile(int(r), int(c)) for r, c in tiles])
@@ -155,7 +158,7 @@ class Plan:
         self._keep = (C.c_double * n_stages)(*[float(v) for v in keep])
         cfg = _Config(C.sizeof(_Config), batch, hidden, n_q_heads, n_kv_heads, head_dim, n_layers,
                       len(tiles), self._tiles, n_stages, self._layers, self._windows, self._keep,
-                      max_text, dtype, xi_mode, engine, int(ragged_input))
+                      max_text, dtype, xi_mode, engine, int(ragged_input), divergence, direction)
         handle = C.c_void_p()
         _check(lib.lightkv_plan(C.byref(cfg), C.byref(handle)), "lightkv_plan")
         self.handle = handle

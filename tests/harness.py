@@ -17,7 +17,8 @@ GAP = 1e-3
 TOL = {"bf16": dict(max_abs=2e-2, rel=1e-2), "fp32": dict(max_abs=None, rel=1e-5)}
 
 
-def prepare_stage(wl, stage, pos=None, dtype="bf16", samples=None, repair=True, tensors=("hidden", "q", "k", "v")):
+def prepare_stage(wl, stage, pos=None, dtype="bf16", samples=None, repair=True, tensors=("hidden", "q", "k", "v"),
+                  metric="cosine", direction="a2b"):
     """Synthetic inputs of one stage with the selection margins enforced on the hidden states."""
     inp = S.make_layer_inputs(wl, stage, pos, dtype=dtype, samples=samples, tensors=tensors)
     rounder = O.to_bf16 if dtype == "bf16" else (lambda a: np.asarray(a, dtype=np.float32).astype(np.float64))
@@ -27,7 +28,8 @@ def prepare_stage(wl, stage, pos=None, dtype="bf16", samples=None, repair=True, 
         for b in range(inp["hidden"].shape[0]):
             nv = int(inp["n_vis"][b])
             fixed, rep = G.enforce_gaps(inp["hidden"][b, vb:vb + nv], inp["pos"][b, :nv], wl.tiles,
-                                        wl.windows[stage], wl.keep[stage], GAP, rounder=rounder)
+                                        wl.windows[stage], wl.keep[stage], GAP, rounder=rounder, metric=metric,
+                                        direction=direction)
             assert rep["ok"], rep
             inp["hidden"][b, vb:vb + nv] = fixed.astype(np.float32)
             reports.append(rep)
@@ -35,14 +37,16 @@ def prepare_stage(wl, stage, pos=None, dtype="bf16", samples=None, repair=True, 
     return inp
 
 
-def oracle_stage(wl, stage, inp, xi_mode="attn", n_text_after=0, text_range=None, text_ranges=None, causal=True):
+def oracle_stage(wl, stage, inp, xi_mode="attn", n_text_after=0, text_range=None, text_ranges=None, causal=True,
+                 metric="cosine", direction="a2b"):
     tb, te = (0, inp["vis_begin"]) if text_range is None else text_range
     q = inp.get("q") if xi_mode in ("attn", "lse") else None
     k = inp.get("k") if xi_mode in ("attn", "lse") else None
     xi = inp.get("xi") if xi_mode == "given" else None
     return O.compress_layer(inp["hidden"], q, k, inp["pos"], inp["n_vis"], inp["vis_begin"], wl.tiles,
                             wl.windows[stage], wl.keep[stage], text_begin=tb, text_end=te, xi=xi,
-                            n_text_after=n_text_after, causal=causal, text_ranges=text_ranges)
+                            n_text_after=n_text_after, causal=causal, text_ranges=text_ranges, metric=metric,
+                            direction=direction)
 
 
 def oracle_lse(inp, n_heads, n_kv, causal=True, n_text_after=0, samples=None):
@@ -85,13 +89,16 @@ def to_device(arr, dtype, device="cuda"):
     return t.to(device)
 
 
-def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_text=None, ragged=False):
+def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_text=None, ragged=False,
+              metric="cosine", direction="a2b"):
     import paper_2605_00789_b200 as L
     xm = {"attn": L.XI_ATTN_FULL, "lse": L.XI_ATTN_LSE, "given": L.XI_GIVEN, "uniform": L.XI_UNIFORM}[xi_mode]
     return L.Plan(batch or wl.batch, wl.hidden, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_layers,
                   wl.tiles, wl.layers, wl.windows, wl.keep, max_text if max_text is not None else wl.n_text + 64,
                   dtype=L.BF16 if dtype == "bf16" else L.FP32, xi_mode=xm,
-                  engine=L.ENGINE_AUTO if engine == "auto" else L.ENGINE_SIMT, ragged_input=ragged)
+                  engine=L.ENGINE_AUTO if engine == "auto" else L.ENGINE_SIMT, ragged_input=ragged,
+                  divergence={"cosine": L.FD_COSINE, "l2sq": L.FD_L2SQ, "l2": L.FD_L2}[metric],
+                  direction=L.DIR_A2B if direction == "a2b" else L.DIR_B2A)
 
 
 def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0, text_range=None,
@@ -276,15 +283,15 @@ def check_lse_out(inp, gpu, n_heads, n_kv, samples, causal=True, n_text_after=0,
 def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge", paged=0, samples=None,
                  stages=None, oracle_samples=None, aux_stream=None, kv_layout="bhnd", kv_stream=None,
                  lse_source="oracle", ragged=False, first_pos=None, text_ranges=None, bidirectional=False,
-                 want_lse=False, expect_status=0):
+                 want_lse=False, expect_status=0, metric="cosine", direction="a2b"):
     """All stages of a workload, chained through the surviving positions; returns per-stage stats.
     first_pos: per-sample positions entering stage 0 (a subset of the grid); ragged: plan built for subsets."""
     bsz = wl.batch if samples is None else len(samples)
-    plan = make_plan(wl, dtype, xi_mode, engine, batch=bsz, ragged=ragged)
+    plan = make_plan(wl, dtype, xi_mode, engine, batch=bsz, ragged=ragged, metric=metric, direction=direction)
     pos = first_pos
     all_stats = []
     for stage in (range(wl.n_stages) if stages is None else stages):
-        inp = prepare_stage(wl, stage, pos, dtype, samples=samples)
+        inp = prepare_stage(wl, stage, pos, dtype, samples=samples, metric=metric, direction=direction)
         if xi_mode == "given":
             rng = np.random.default_rng(stage)
             inp["xi"] = rng.uniform(0.05, 3.0, size=inp["pos"].shape).astype(np.float32)
@@ -298,7 +305,8 @@ def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge
         osamp = list(range(bsz)) if oracle_samples is None else oracle_samples
         sub = {key: (val[osamp] if isinstance(val, np.ndarray) and val.shape[:1] == (bsz,) else val)
                for key, val in inp.items()}
-        ref = oracle_stage(wl, stage, sub, xi_mode, text_ranges=text_ranges, causal=not bidirectional)
+        ref = oracle_stage(wl, stage, sub, xi_mode, text_ranges=text_ranges, causal=not bidirectional,
+                           metric=metric, direction=direction)
         stats = compare_stage(wl, stage, inp, ref, gpu, dtype, kv_mode, samples=osamp, expect_status=expect_status)
         if want_lse:
             check_lse_out(inp, gpu, wl.n_q_heads, wl.n_kv_heads, osamp, causal=not bidirectional)

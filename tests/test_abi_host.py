@@ -37,7 +37,7 @@ def test_struct_layouts_match_the_header(L, tmp_path):
 #include <stddef.h>
 #include "lightkv.h"
 int main(void) {
-  printf("%zu %zu\\n", sizeof(lightkv_config_t), offsetof(lightkv_config_t, ragged_input));
+  printf("%zu %zu\\n", sizeof(lightkv_config_t), offsetof(lightkv_config_t, direction));
   printf("%zu %zu\\n", sizeof(lightkv_stage_info_t), offsetof(lightkv_stage_info_t, reserved));
   printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, lse_out_head_stride));
   printf("%zu %zu\\n", sizeof(lightkv_kv_args_t), offsetof(lightkv_kv_args_t, stream));
@@ -48,7 +48,7 @@ int main(void) {
     subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
     rows = [tuple(int(v) for v in line.split()) for line in subprocess.check_output([str(exe)]).decode().splitlines()]
     k = L.lightkv
-    got = [(C.sizeof(k._Config), k._Config.ragged_input.offset),
+    got = [(C.sizeof(k._Config), k._Config.direction.offset),
            (C.sizeof(k._StageInfo), k._StageInfo.reserved.offset),
            (C.sizeof(k._LayerArgs), k._LayerArgs.lse_out_head_stride.offset),
            (C.sizeof(k._KvArgs), k._KvArgs.stream.offset)]
@@ -86,7 +86,7 @@ def test_plan_counts_and_retention(L):
     dict(batch=0), dict(hidden=65), dict(head_dim=12), dict(n_q_heads=3), dict(keep=[0.4, 0.5]),
     dict(keep=[0.5, 1.5]), dict(windows=[7, 1]), dict(windows=[0, 1]), dict(layers=[4, 2]),
     dict(layers=[2, 9]), dict(tiles=[(0, 6)]), dict(dtype=7), dict(xi_mode=9), dict(engine=5),
-    dict(ragged_input=2),
+    dict(ragged_input=2), dict(divergence=3), dict(direction=2),
 ])
 def test_plan_rejects_bad_configs(L, kw):
     with pytest.raises(L.LightKVError, match="invalid argument"):

@@ -231,6 +231,47 @@ def test_the_librarys_own_row_lse_feeds_the_lse_mode(name):
     np.testing.assert_allclose(a["xi_out"][:, :nv], b["xi_out"][:, :nv], rtol=2e-3)
 
 
+@pytest.mark.parametrize("name", ["small", "cfg1"])
+def test_logits_far_above_the_first_tiles_maximum_take_the_safe_pass(name):
+    """The tensor-core xi kernel subtracts the maximum of a row's FIRST key tile and checks its sums at the end.
+    Here one late key of one KV head is scaled by 128, so that many rows meet a logit far more than 88 above
+    that reference: their sums leave the fp32 range, the CTA repeats the item with a running maximum, and the
+    result still matches the oracle (the other heads keep xi away from zero)."""
+    wl = S.workload(name)
+    plan = H.make_plan(wl)
+    inp = H.prepare_stage(wl, 0)
+    late = inp["vis_begin"] + int(inp["n_vis"].min()) * 2 // 3
+    inp["k"][:, 0, late] *= 128.0                              # a power of two: still bf16 values
+    logit = inp["q"][0, 0, late + 1:] @ inp["k"][0, 0, late] / np.sqrt(wl.head_dim)
+    first = (inp["q"][0, 0, late + 1:] @ inp["k"][0, 0, :64].T / np.sqrt(wl.head_dim)).max(axis=1)
+    assert (logit - first > 100).any()                         # the case really leaves the fp32 range
+    gpu = H.gpu_stage(plan, wl, 0, inp, want_lse=True)
+    del gpu["k_out"], gpu["v_out"]      # the scaled key row is outside the value range the bf16 K/V tolerance is meant for
+    H.compare_stage(wl, 0, inp, H.oracle_stage(wl, 0, inp), gpu)
+    H.check_lse_out(inp, gpu, wl.n_q_heads, wl.n_kv_heads, range(inp["hidden"].shape[0]), atol=2e-2)
+    plan.close()
+
+
+# ---- the variants the paper ablates: Euclidean pair scores, reverse message direction ---------------------------
+
+@pytest.mark.parametrize("metric", ["l2sq", "l2"])
+@pytest.mark.parametrize("dtype,engine", [("bf16", "auto"), ("bf16", "simt"), ("fp32", "simt")])
+def test_euclidean_pair_scores(metric, dtype, engine):
+    H.run_schedule(S.workload("small"), dtype=dtype, engine=engine, metric=metric)
+    if dtype == "bf16" and metric == "l2sq":
+        H.run_schedule(S.workload("cfg1"), engine=engine, metric=metric)      # windows of 36 / 72 / 144 tokens
+
+
+@pytest.mark.parametrize("engine", ["simt", "auto"])
+def test_reverse_direction_b_into_a(engine):
+    # odd windows: the destinations (A) outnumber the sources (B); keep 0.5 on even windows removes all of B
+    H.run_schedule(S.workload("small"), engine=engine, direction="b2a")
+    H.run_schedule(S.workload("tiny"), engine=engine, direction="b2a", xi_mode="given")
+    stats = H.run_schedule(S.workload("cfg1"), engine=engine, direction="b2a")
+    assert [s["n_out"] for s in stats] == [[288], [144], [72]]
+    H.run_schedule(S.workload("cfg1r"), engine=engine, direction="b2a", metric="l2sq", stages=[0, 1])
+
+
 # ---- persistent CTAs that take more than one work item ---------------------------------------------------------
 
 def _sm_count():
@@ -259,10 +300,11 @@ def test_cfg2_lse_mode_full_size_sampled():
 
 @pytest.mark.parametrize("hidden,ragged", [(64, False), (72, True)])
 def test_fd_persistent_ctas_take_several_tiles(hidden, ragged):
-    # 48 samples x 36 windows of 16 tokens: eight tiles per sample, 384 tiles for the 2 x SMs persistent CTAs of
-    # the tensor-core FD kernel, so CTAs loop over tiles (ring phases and the accumulator barrier run on); the
-    # ragged variant gives every sample its own subset of the grid under a plan built for subsets
-    wl = S.Workload(name="fdmulti", config_id=131, batch=48, tiles=((24, 24),), n_text=4, hidden=hidden,
+    # 160 samples x 36 windows of 16 tokens: three tiles of sixteen windows per sample (a tile holds at most 128 A
+    # nodes), 480 tiles for the 2 x SMs persistent CTAs of the tensor-core FD kernel, so most CTAs take a second
+    # tile (ring phases and the accumulator barrier run on); the ragged variant gives every sample its own subset
+    # of the grid under a plan built for subsets
+    wl = S.Workload(name="fdmulti", config_id=131, batch=160, tiles=((24, 24),), n_text=4, hidden=hidden,
                     n_q_heads=2, n_kv_heads=1, head_dim=64, n_layers=16, layers=(3,), windows=(6,), keep=(0.5,))
     first = None
     if ragged:
@@ -270,7 +312,7 @@ def test_fd_persistent_ctas_take_several_tiles(hidden, ragged):
         full = np.arange(wl.n_vis, dtype=np.int32)
         first = [np.sort(rng.choice(full, int(rng.integers(500, 577)), replace=False)).astype(np.int32)
                  for _ in range(wl.batch)]
-    stats = H.run_schedule(wl, xi_mode="uniform", oracle_samples=[0, 17, 47], ragged=ragged, first_pos=first)
+    stats = H.run_schedule(wl, xi_mode="uniform", oracle_samples=[0, 17, 159], ragged=ragged, first_pos=first)
     info = stats[0]["info"]
     assert info.uses_tensor_cores == 1 and info.fd_tiles * wl.batch > 2 * _sm_count()
 

@@ -171,6 +171,18 @@ def _scaled_logits_always_causal(q, k, vis_begin, n_vis, causal=True):
     return O_scaled_logits(q, k, vis_begin, n_vis, True)
 
 
+def _divergence_l2sq_without_the_cross_term(xa, xb, metric="cosine"):
+    if metric == "cosine":
+        return O_divergence(xa, xb, metric)
+    xa, xb = np.asarray(xa, dtype=F64), np.asarray(xb, dtype=F64)
+    sq = (xa * xa).sum(axis=1)[:, None] + (xb * xb).sum(axis=1)[None, :]
+    return sq if metric == "l2sq" else np.sqrt(sq)
+
+
+def _compress_vision_ignores_the_direction(x, pos, xi, tiles, w, keep, metric="cosine", direction="a2b"):
+    return O_compress_vision(x, pos, xi, tiles, w, keep, metric, "a2b")
+
+
 def _window_of_swapped_axes(pos, tiles, w):
     return O_window_of(pos, [(c, r) for r, c in tiles], w)
 
@@ -187,6 +199,7 @@ O_feature_divergence, O_removal_count, O_xi_from_attention = O.feature_divergenc
 O_attention_rows, O_message_passing, O_window_of = O.attention_rows, O.message_passing, O.window_of
 O_retention, O_compact_kv = O.retention, O.compact_kv
 O_row_logsumexp, O_scaled_logits = O.row_logsumexp, O.scaled_logits
+O_divergence, O_compress_vision = O.divergence, O.compress_vision
 
 MUTATIONS = [
     ("feature_divergence", _fd_wrong_sign),
@@ -208,6 +221,8 @@ MUTATIONS = [
     ("row_logsumexp", _row_logsumexp_without_the_scale),
     ("xi_from_attention", _xi_first_range_only),
     ("scaled_logits", _scaled_logits_always_causal),
+    ("divergence", _divergence_l2sq_without_the_cross_term),
+    ("compress_vision", _compress_vision_ignores_the_direction),
     ("window_of", _window_of_swapped_axes),
     ("retention", _retention_counts_the_compression_layer_as_compressed),
     ("compact_kv", _compact_kv_ignores_the_weights),

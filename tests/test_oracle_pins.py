@@ -153,6 +153,24 @@ def test_bipartition_parity():
     assert list(a) == [10, 12, 14] and list(b) == [11, 13]     # 1st, 3rd, 5th -> A
 
 
+def test_euclidean_divergences_against_the_library():
+    # appendix "Influence of similarity metrics": squared and plain Euclidean distance as the pair score
+    import scipy.spatial.distance as D
+    rng = np.random.default_rng(21)
+    xa, xb = rng.standard_normal((5, 7)), rng.standard_normal((4, 7))
+    np.testing.assert_allclose(O.divergence(xa, xb, "l2sq"), D.cdist(xa, xb, "sqeuclidean"), rtol=1e-13)
+    np.testing.assert_allclose(O.divergence(xa, xb, "l2"), D.cdist(xa, xb, "euclidean"), rtol=1e-13)
+    np.testing.assert_array_equal(O.divergence(xa, xb, "cosine"), O.feature_divergence(xa, xb))
+    # on unit vectors the squared distance is twice the feature divergence
+    ua, ub = xa / np.linalg.norm(xa, axis=1, keepdims=True), xb / np.linalg.norm(xb, axis=1, keepdims=True)
+    np.testing.assert_allclose(O.divergence(ua, ub, "l2sq"), 2.0 * O.feature_divergence(ua, ub), rtol=1e-12, atol=1e-15)
+    # unlike FD it is not scale invariant: a long vector is far from everything
+    far = O.divergence(10.0 * xa[:1], xb, "l2sq")
+    assert (far > O.divergence(xa[:1], xb, "l2sq")).all()
+    with pytest.raises(ValueError):
+        O.divergence(xa, xb, "manhattan")
+
+
 # ------------------------------------------------------------------ xi (Eq. "attention-factor")
 
 def _rand_qk(rng, n_heads, n_kv, n_seq, dh):
@@ -356,6 +374,31 @@ def test_direction_is_a_into_b_and_position_of_group_is_b():
     np.testing.assert_array_equal(res["pos_out"], np.arange(1, 36, 2))
     assert (res["partner"][0::2] % 2 == 1).all() and (res["partner"][1::2] == -1).all()
     assert (np.diff(res["pos_out"]) > 0).all()
+
+
+def test_reverse_direction_is_the_forward_one_on_the_mirrored_window():
+    """B -> A: the two sets swap roles.  Exchanging the contents of positions (0,1), (2,3), ... turns every A node
+    into a B node and back, so the reverse direction on the exchanged window merges exactly the same tokens into
+    exactly the same rows as the forward direction on the original."""
+    x, pos, xi, tiles, w, keep = _case(23, keep=0.7)
+    swap = np.arange(len(x)) ^ 1
+    fwd = O.compress_vision(x, pos, xi, tiles, w, keep)
+    rev = O.compress_vision(x[swap], pos, xi[swap], tiles, w, keep, direction="b2a")
+    # token t of the exchanged window is token t ^ 1 of the original
+    np.testing.assert_array_equal(rev["partner"][swap] >= 0, fwd["partner"] >= 0)
+    merged = np.nonzero(fwd["partner"] >= 0)[0]
+    np.testing.assert_array_equal(rev["partner"][merged ^ 1] ^ 1, fwd["partner"][merged])
+    np.testing.assert_allclose(rev["weight"][swap], fwd["weight"], rtol=1e-14)
+    by_survivor_f = {int(s): fwd["x_out"][o] for o, s in enumerate(fwd["survivor"])}
+    by_survivor_r = {int(s) ^ 1: rev["x_out"][o] for o, s in enumerate(rev["survivor"])}
+    assert sorted(by_survivor_f) == sorted(by_survivor_r)
+    for s_ in by_survivor_f:
+        np.testing.assert_allclose(by_survivor_r[s_], by_survivor_f[s_], rtol=1e-13, atol=1e-15)
+    # sources are the B nodes: an odd window can lose at most floor(n / 2) tokens, and all survivors of keep = 0.5 are A
+    xo, poso, xio = x[:35], pos[:35], xi[:35]
+    half = O.compress_vision(xo, poso, xio, [(5, 7)], 1, 0.5, direction="b2a")
+    assert int(half["n_out"]) == 18 and (half["pos_out"] % 2 == 0).all()
+    assert (half["partner"][1::2] % 2 == 0).all() and (half["partner"][0::2] == -1).all()
 
 
 def test_keep_one_is_identity():
