@@ -56,6 +56,8 @@ struct Workspace {
   int* partner;    // [B, cap_in]         token an A token is merged into, -1 = survives
   int* slot;       // [B, cap_in]         output slot of surviving tokens
   int* a_partner;  // [B, cap_a]          per A entry: token it is merged into, -1 = survives
+  unsigned int* xi_sched;   // [4]        ticket counters and list length of the tensor-core xi kernel
+  int* xi_redo;    // [ceil(cap_in / 128) * H * B]  its work items that need the second, safe launch
   int cap_in, cap_out, cap_a, cap_b, n_windows;
 };
 

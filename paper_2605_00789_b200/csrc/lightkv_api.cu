@@ -20,7 +20,7 @@ struct StagePlan {
   int fd_tiles;    // estimate of the tiles per sample of the tensor-core FD kernel (sizes its launch)
   Geometry geo;
   size_t ws_bytes;
-  size_t off[14];     // byte offsets of the Workspace arrays
+  size_t off[16];     // byte offsets of the Workspace arrays
 };
 
 }  // namespace lkv
@@ -53,13 +53,14 @@ static int fd_tile_count(int n_windows, int max_a, int batch) {
 static void layout_workspace(const lightkv_plan_t& p, StagePlan& s) {
   const size_t B = p.cfg.batch, nW1 = s.n_windows + 1;
   const bool attn = p.cfg.xi_mode == LIGHTKV_XI_ATTN_FULL || p.cfg.xi_mode == LIGHTKV_XI_ATTN_LSE;
-  const size_t sizes[14] = {
+  const size_t xi_items = attn ? size_t((s.cap_in + 127) / 128) * p.cfg.n_q_heads * B : 0;
+  const size_t sizes[16] = {
       B * nW1 * 4, B * nW1 * 4, B * s.cap_in * 4, B * s.cap_in * 4, B * s.cap_a * 4, B * s.cap_a * 4,
       B * s.cap_b * 4, B * s.cap_a * 8, B * sizeof(FdTiling),
       attn ? B * p.cfg.n_q_heads * s.cap_in * 4 : 0, B * s.cap_in * 4, B * s.cap_in * 4, B * s.cap_in * 4,
-      B * s.cap_a * 4};
+      B * s.cap_a * 4, attn ? size_t(16) : size_t(0), xi_items * 4};
   size_t off = 0;
-  for (int i = 0; i < 14; ++i) { s.off[i] = off; off += align_up(sizes[i], 256); }
+  for (int i = 0; i < 16; ++i) { s.off[i] = off; off += align_up(sizes[i], 256); }
   s.ws_bytes = std::max<size_t>(off, 256);
 }
 
@@ -80,6 +81,8 @@ static Workspace bind_workspace(const StagePlan& s, void* base) {
   w.partner = reinterpret_cast<int*>(p + s.off[11]);
   w.slot = reinterpret_cast<int*>(p + s.off[12]);
   w.a_partner = reinterpret_cast<int*>(p + s.off[13]);
+  w.xi_sched = reinterpret_cast<unsigned int*>(p + s.off[14]);
+  w.xi_redo = reinterpret_cast<int*>(p + s.off[15]);
   w.cap_in = s.cap_in; w.cap_out = s.cap_out; w.cap_a = s.cap_a; w.cap_b = s.cap_b;
   w.n_windows = s.n_windows;
   return w;

@@ -48,26 +48,31 @@ static bool make_map_bhnd(CUtensorMap* map, const void* base, int width, int row
 // ======================================================================================================
 // xi per head on tensor cores (Eq. "attention-factor" over the softmax rows of Eq. "attention-matrix").
 //
-// A work item is (tile of 128 vision queries, head, sample); three CTAs share an SM.  Warp 0 streams the Q
-// tile once and the K tiles (64 keys) through a 2-stage ring with TMA; warp 1 issues S = Q K^T (128 x 64 x dh,
-// bf16 -> fp32) into one of two TMEM accumulators; warps 2-5 own one query row per thread (= TMEM lane), pull
-// the 64 logits of the row into registers, release the accumulator, and add exp(logit - reference) to two
-// sums per row (all visible keys / prompt keys J).  Output per head: sum_J / sum_all.
+// A work item is (tile of 128 vision queries, head, sample).  Persistent CTAs, two per SM, draw items from a
+// ticket counter in global memory (items of one head are neighbours in the list, so concurrent CTAs share
+// its K in L2; within a head the longest rows come first).  Warp 0 is the scheduler and the TMA producer: it
+// publishes the ticket to the other roles through a two-slot ring in shared memory, streams the item's Q tile
+// once and its K tiles (128 keys) through a 2-stage ring; the next item's Q and first K tiles are requested as
+// soon as the MMAs of the current item have drained, i.e. while its last tiles are still in the softmax warps.
+// Warp 1 issues S = Q K^T (128 x 128 x dh, bf16 -> fp32) into one of two TMEM accumulators.  Warps 2-5 own one
+// query row per thread (= TMEM lane): they pull the accumulator into registers in two halves of 64 logits,
+// release it, and add exp(logit - reference) to two sums per row (all visible keys / prompt keys J).
+// Output per head: sum_J / sum_all.
 //
 // The kernel is bound by the exponentials (one per logit on the special-function unit, 16 per clock per SM,
 // against one MMA per tile), so the softmax arithmetic is kept to three instructions per logit:
-//   * the reference subtracted before the exponential is the row's maximum over the FIRST key tile only
+//   * the reference subtracted before the exponential is the row's maximum over the FIRST 64 keys only
 //     (softmax is invariant to the reference; fp32 holds exp of any later logit up to 88 above it), so the
 //     other tiles need no maximum and no rescaling;
-//   * on tiles that need neither the causal mask nor the prompt mask, every fourth exponential is evaluated
+//   * on halves that need neither the causal mask nor the prompt mask, every fourth exponential is evaluated
 //     on the FMA pipe instead (range reduction + cubic, relative error 7.5e-5), which takes a quarter of the
 //     load off the special-function unit.
-// A row whose sum left the fp32 range (a later logit more than 88 above the first tile's maximum) is found at
-// the end of the item: the CTA then repeats the item with a running maximum and rescaling, as an ordinary
-// online softmax does, and overwrites its results.  Tiles that straddle the diagonal (or the end of the
-// sample) are masked, and the columns no row of a warp can see are skipped.
-// With the caller's row log-sum-exp (WALK) only the prompt key tiles are visited and the CTAs walk the item
-// list, so that an item's loads overlap the previous item's arithmetic.
+// A row whose sum left the fp32 range (a later logit more than 88 above the first keys' maximum) is found at
+// the end of its item, which is then appended to a list in global memory; a second launch of the kernel
+// (SAFE) walks that list with a running maximum and rescaling on every half, as an ordinary online softmax
+// does, and overwrites the item's results.  With an empty list that launch returns at once.
+// Halves that straddle the diagonal (or the end of the sample) are masked, and the columns no row of a warp
+// can see are skipped.  With the caller's row log-sum-exp (LSE) only the prompt key tiles are visited.
 // ======================================================================================================
 __device__ __forceinline__ float ex2(float x) {          // one MUFU op, flush-to-zero
   float y;
@@ -87,6 +92,14 @@ __device__ __forceinline__ float ex2_fma(float x) {
   return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
 
+// Scheduler words in the workspace (zeroed on the stream before the first launch of a call).
+struct XiSched {
+  unsigned int ticket;               // next item of the first launch
+  unsigned int safe_ticket;          // next entry of the list, second launch
+  unsigned int n_redo;               // items appended to the list
+  unsigned int pad;
+};
+
 struct XiTcArgs {
   const int* n_vis;
   float* xi_h;
@@ -100,81 +113,95 @@ struct XiTcArgs {
   int cap_in, vis_begin, n_q_heads, group;
   int batch, n_qt;                   // samples, query tiles of 128 rows per (sample, head)
   float scale2;                      // log2(e) / sqrt(dh)
+  XiSched* sched;
+  int* redo_list;                    // [n_qt * H * B] items whose sums left the fp32 range
 };
 
-constexpr int XT_STAGES = 2;
-constexpr int XT_KEY_TILE = 64;      // keys per tile: two 64-column accumulators per CTA, three CTAs per SM
+constexpr int XT_STAGES = 2;         // K tiles in the shared-memory ring
+constexpr int XT_SBUF = 2;           // S accumulators in tensor memory
+constexpr int XT_CTAS = 2;           // CTAs per SM
+constexpr int XT_KEY_TILE = 128;     // keys per K tile and per MMA (the softmax warps read it as two halves of 64)
+constexpr int XT_SUB = 64;           // keys per half
+constexpr int XT_THREADS = 320;      // TMA / scheduler warp, MMA warp, eight softmax warps
+constexpr int XT_HEAD_GROUP = 64;    // (sample, head) pairs whose work items are interleaved (their K: 64 x ~1 MB)
 
-// WALK = true <=> the caller supplied the row log-sum-exp (a.lse != nullptr).
-template <int DH, int BK, bool WALK>
-__global__ void __launch_bounds__(192, 3)
+// LSE: the caller supplied the row log-sum-exp (a.lse != nullptr).  SAFE: second launch, items from the list.
+template <int DH, bool LSE, bool SAFE>
+__global__ void __launch_bounds__(XT_THREADS, XT_CTAS)
 xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, XiTcArgs a) {
   grid_dependency_sync();
-  static_assert(BK == 64, "the prompt mask of a tile is one 64-bit word");
+  constexpr int BK = XT_KEY_TILE;
+  static_assert(BK == 2 * XT_SUB && XT_SUB == 64, "a K tile is two halves of 64 keys; the prompt mask of a half is one 64-bit word");
+  static_assert(!(LSE && SAFE), "with the caller's normaliser no sum can leave the fp32 range");
   constexpr int HALVES = DH / 64;
   constexpr uint32_t TILE_BYTES = HALVES * 16384;          // Q tile: 128 rows x DH bf16
   constexpr uint32_t KHALF_BYTES = BK * 128;               // BK key rows x 64 columns
   constexpr uint32_t KT_BYTES = HALVES * KHALF_BYTES;      // K tile: BK rows x DH bf16
-  constexpr int NC = BK / 32;                              // 32-column chunks of a tile
-  constexpr int N_PASS = WALK ? 1 : 2;                     // second pass: the item again, with a running maximum
+  const unsigned int n_items = SAFE ? a.sched->n_redo : unsigned(a.n_qt) * a.n_q_heads * a.batch;
+  if (n_items == 0) return;                                // nothing on the list: the usual case of the second launch
+
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* q_s = base;
   unsigned char* k_s = base + TILE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + TILE_BYTES + KT_BYTES * XT_STAGES);
   uint64_t* q_full = bars;
-  uint64_t* k_full = bars + 1;                 // [XT_STAGES]
+  uint64_t* q_empty = bars + 1;                // every MMA that reads the Q tile has completed
+  uint64_t* k_full = bars + 2;                 // [XT_STAGES]
   uint64_t* k_empty = k_full + XT_STAGES;      // [XT_STAGES]
-  uint64_t* s_full = k_empty + XT_STAGES;      // [2]
-  uint64_t* s_empty = s_full + 2;              // [2]
-  uint64_t* q_empty = s_empty + 2;             // every MMA that reads the Q tile has completed
-  uint64_t* verdict = q_empty + 1;             // the four softmax warps have checked their sums of the first pass
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(verdict + 1);
+  uint64_t* s_full = k_empty + XT_STAGES;      // [XT_SBUF]
+  uint64_t* s_empty = s_full + XT_SBUF;        // [XT_SBUF]
+  uint64_t* item_full = s_empty + XT_SBUF;     // [2] the scheduler published an item
+  uint64_t* item_empty = item_full + 2;        // [2] the MMA thread and the eight softmax warps have read it
+  uint64_t* pair_full = item_empty + 2;        // the upper column group has stored its partial sums of an item
+  uint64_t* pair_empty = pair_full + 1;        // the lower column group has read them
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pair_empty + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* redo = const_cast<int*>(abort_flag) + 1;            // some row's sum left the fp32 range
+  volatile int* item_slot = abort_flag + 1;    // [2]
+  int* redo_mark = const_cast<int*>(item_slot) + 2;      // last item this CTA put on the list
+  float* pair_m = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(bars) + 256);   // [128] each
+  float* pair_all = pair_m + 128;
+  float* pair_txt = pair_all + 128;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // Work items: (query tile, head, sample), the query tiles of one head next to each other (they share its K
-  // in L2), longest rows first.  WALK = false: one item per CTA, grid (query tiles, heads, samples).
-  // WALK = true: CTA c takes items c, c + gridDim.x, ... of the flattened list; every role walks the list
-  // with the same tests, so their barrier phases stay in step.
-  const int n_items = WALK ? a.n_qt * a.n_q_heads * a.batch : 0;
   // key tiles to visit: all tiles up to the last query's own key, or, when the caller supplies the row
   // log-sum-exp, only the tiles that hold prompt keys (J lies before the vision block, so it is visible)
-  const int kt_lo = WALK ? a.text.begin / BK : 0;
+  const int kt_lo = LSE ? a.text.begin / BK : 0;
   const int nkt_lse = a.text.end > a.text.begin ? (a.text.end - 1) / BK + 1 - kt_lo : 0;
-  struct Item { int h, b, t0, nq, s_first, nkt, n_seq; };
+  struct Item { int h, b, t0, nq, s_first, nkt, n_seq, nsub; };   // nsub: halves of 64 keys the item visits
+  // item -> (query tile, head, sample).  The (sample, head) pairs are taken in groups of XT_HEAD_GROUP whose keys
+  // stay in L2 together; inside a group the list runs over the query tiles from the longest rows to the shortest,
+  // all pairs of the group for each, so that the work left for the last tickets is short.
   auto decode = [&](int item, Item& it) -> bool {
-    int qt;
-    if (WALK) {
-      const int hb = item / a.n_qt;
-      qt = a.n_qt - 1 - item % a.n_qt; it.h = hb % a.n_q_heads; it.b = hb / a.n_q_heads;
-    } else {
-      qt = gridDim.x - 1 - blockIdx.x; it.h = blockIdx.y; it.b = blockIdx.z;
-    }
+    const int n_hb = a.n_q_heads * a.batch, per_group = XT_HEAD_GROUP * a.n_qt;
+    const int grp = item / per_group, within = item - grp * per_group;
+    const int gsize = min(XT_HEAD_GROUP, n_hb - grp * XT_HEAD_GROUP);
+    const int hb = grp * XT_HEAD_GROUP + within % gsize, qt = a.n_qt - 1 - within / gsize;
+    it.h = hb % a.n_q_heads; it.b = hb / a.n_q_heads;
     const int n = a.n_vis ? min(a.n_vis[it.b], a.cap_in) : a.cap_in;
     it.t0 = qt * 128;
     if (it.t0 >= n) return false;
     it.nq = min(128, n - it.t0);
     it.s_first = a.vis_begin + it.t0;
     it.n_seq = a.vis_begin + n + a.n_text_after;
-    it.nkt = WALK ? nkt_lse : ((a.bidirectional ? it.n_seq : it.s_first + it.nq) - 1) / BK + 1;
+    it.nsub = LSE ? 2 * nkt_lse : ((a.bidirectional ? it.n_seq : it.s_first + it.nq) - 1) / XT_SUB + 1;
+    it.nkt = (it.nsub + 1) / 2;
     return true;
   };
-  Item it0 = {};
-  if (!WALK && !decode(0, it0)) return;        // one item per CTA: decoded once, before the set-up
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
-    mbar_init(verdict, 4);
     for (int i = 0; i < XT_STAGES; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4); }
+    for (int i = 0; i < XT_SBUF; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 8); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 9); }
+    mbar_init(pair_full, 4);
+    mbar_init(pair_empty, 4);
     *abort_flag = 0;
-    *redo = 0;
+    *redo_mark = -1;
     fence_barrier_init();
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, 2 * BK); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(tmem_slot, XT_SBUF * BK); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -182,201 +209,246 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {
+      // ---- scheduler + TMA producer
       prefetch_tensormap(&q_map);
       prefetch_tensormap(&k_map);
-      uint32_t kf = 0, done = 0;                       // K tiles fetched / items started by this CTA
-      bool ok = true;
-      for (int item = blockIdx.x; ok && (!WALK || item < n_items); item += gridDim.x) {
-        Item it = it0;
-        if ((WALK && !decode(item, it)) || it.nkt == 0) { if (WALK) continue; else break; }
-        for (int pass = 0; ok && pass < N_PASS; ++pass) {
-          if (pass == 1 && (!mbar_wait(verdict, 0, abort_flag) || !*redo)) break;
-          if (pass == 0) {
-            // the Q tile is free once every MMA of the previous item has completed
-            if (WALK && done > 0 && !mbar_wait(q_empty, (done - 1) & 1, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(q_full, TILE_BYTES);
+      uint32_t kf = 0, n = 0, nq_loaded = 0;           // K tiles fetched / items published / Q tiles loaded
+      for (;;) {
+        const uint32_t slot = n & 1;
+        if (!mbar_wait(&item_empty[slot], ((n >> 1) & 1) ^ 1, abort_flag)) break;
+        const unsigned int t = atomicAdd(SAFE ? &a.sched->safe_ticket : &a.sched->ticket, 1u);
+        const int item = t < n_items ? (SAFE ? a.redo_list[t] : int(t)) : -1;
+        item_slot[slot] = item;
+        mbar_arrive(&item_full[slot]);                 // release: the slot is written before the arrival is seen
+        ++n;
+        if (item < 0) break;
+        Item it;
+        if (!decode(item, it) || it.nkt == 0) continue;
+        // the Q tile is free once every MMA of the previous item has completed
+        if (nq_loaded > 0 && !mbar_wait(q_empty, (nq_loaded - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(q_full, TILE_BYTES);
 #pragma unroll
-            for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.s_first, it.h, it.b);
-          }
-          const int hk = it.h / a.group;
-          for (int kt = 0; kt < it.nkt; ++kt, ++kf) {
-            const uint32_t s = kf % XT_STAGES;
-            if (!mbar_wait(&k_empty[s], ((kf / XT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(&k_full[s], KT_BYTES);
+        for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.s_first, it.h, it.b);
+        ++nq_loaded;
+        const int hk = it.h / a.group;
+        bool ok = true;
+        for (int kt = 0; kt < it.nkt; ++kt, ++kf) {
+          const uint32_t s = kf % XT_STAGES;
+          if (!mbar_wait(&k_empty[s], ((kf / XT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(&k_full[s], KT_BYTES);
 #pragma unroll
-            for (int hf = 0; hf < HALVES; ++hf)
-              tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, it.b);
-          }
+          for (int hf = 0; hf < HALVES; ++hf)
+            tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, it.b);
         }
-        ++done;
-        if (!WALK) break;
+        if (!ok) break;
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(128, BK);
-      const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s);
-      uint32_t kc = 0, done = 0;                       // K tiles consumed / items started
-      bool ok = true;
-      for (int item = blockIdx.x; ok && (!WALK || item < n_items); item += gridDim.x) {
-        Item it = it0;
-        if ((WALK && !decode(item, it)) || it.nkt == 0) { if (WALK) continue; else break; }
-        for (int pass = 0; ok && pass < N_PASS; ++pass) {
-          if (pass == 1 && (!mbar_wait(verdict, 0, abort_flag) || !*redo)) break;
-          if (pass == 0 && !mbar_wait(q_full, done & 1, abort_flag)) { ok = false; break; }
-          for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
-            const uint32_t s = kc % XT_STAGES, buf = kc & 1;
-            if (!mbar_wait(&s_empty[buf], ((kc >> 1) & 1) ^ 1, abort_flag) ||
-                !mbar_wait(&k_full[s], (kc / XT_STAGES) & 1, abort_flag)) { ok = false; break; }
-            tc_fence_after();
+      // ---- MMA issue
+      constexpr uint32_t idesc_full = idesc_bf16(128, BK), idesc_half = idesc_bf16(128, XT_SUB);
+      // the operand descriptors are built once (Q: one per 16-column step; K: those of ring stage 0, a stage
+      // adds a constant to the address field)
+      uint64_t q_desc[DH / 16], k_desc[DH / 16];
 #pragma unroll
-            for (int kk = 0; kk < DH / 16; ++kk) {
-              umma_bf16(tmem_base + buf * BK, smem_desc_sw128(q_addr + (kk >> 2) * 16384 + (kk & 3) * 32),
-                        smem_desc_sw128(k_addr + s * KT_BYTES + (kk >> 2) * KHALF_BYTES + (kk & 3) * 32), idesc, kk > 0);
-            }
-            umma_commit(&k_empty[s]);
-            umma_commit(&s_full[buf]);
-          }
+      for (int kk = 0; kk < DH / 16; ++kk) {
+        q_desc[kk] = smem_desc_sw128(smem_u32(q_s) + (kk >> 2) * 16384 + (kk & 3) * 32);
+        k_desc[kk] = smem_desc_sw128(smem_u32(k_s) + (kk >> 2) * KHALF_BYTES + (kk & 3) * 32);
+      }
+      uint32_t kc = 0, n = 0, nq_used = 0;             // K tiles consumed / items read / Q tiles used
+      for (;;) {
+        const uint32_t slot = n & 1;
+        if (!mbar_wait(&item_full[slot], (n >> 1) & 1, abort_flag)) break;
+        const int item = item_slot[slot];
+        mbar_arrive(&item_empty[slot]);
+        ++n;
+        if (item < 0) break;
+        Item it;
+        if (!decode(item, it) || it.nkt == 0) continue;
+        if (!mbar_wait(q_full, nq_used & 1, abort_flag)) break;
+        bool ok = true;
+        for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
+          const uint32_t s = kc % XT_STAGES, buf = kc % XT_SBUF;
+          if (!mbar_wait(&s_empty[buf], ((kc / XT_SBUF) & 1) ^ 1, abort_flag) ||
+              !mbar_wait(&k_full[s], (kc / XT_STAGES) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t stage_off = uint64_t(s * (KT_BYTES >> 4));     // the address field counts 16-byte units
+          const uint32_t d_addr = tmem_base + buf * BK;
+          // the last tile of an odd number of halves needs its first 64 keys only
+          const uint32_t idesc = (2 * kt + 2 > it.nsub) ? idesc_half : idesc_full;
+#pragma unroll
+          for (int kk = 0; kk < DH / 16; ++kk) umma_bf16(d_addr, q_desc[kk], k_desc[kk] + stage_off, idesc, kk > 0);
+          umma_commit(&k_empty[s]);
+          umma_commit(&s_full[buf]);
         }
-        if (WALK && ok) umma_commit(q_empty);
-        ++done;
-        if (!WALK) break;
+        if (!ok) break;
+        umma_commit(q_empty);
+        ++nq_used;
       }
     }
   } else {
-    const int quad = warp & 3;                          // TMEM lanes this warp may read
+    // ---- softmax warps: two threads per query row.  Warps 2-5 take the lower 32 columns of every half of 64
+    //      keys, warps 6-9 the upper 32; warp w may read the TMEM lanes of quadrant w % 4.  Each thread keeps
+    //      its own reference and sums; the two partial results of a row are combined once per item.
+    const int sw = warp - 2, quad = warp & 3, cg = sw >> 2;   // softmax warp 0..7, lane quadrant, column group
     const int r = quad * 32 + lane;                     // query row of this thread
-    const uint32_t lane_addr = tmem_base + (uint32_t(quad * 32) << 16);
+    const uint32_t lane_addr = tmem_base + (uint32_t(quad * 32) << 16) + cg * 32;
     const float sc = a.scale2;
-    uint32_t kc = 0;                                    // key tiles consumed by this CTA so far
+    uint32_t kc = 0, n = 0, np = 0;                     // key tiles consumed / items read / exchanges done by this CTA
     bool alive = true;
-    for (int item = blockIdx.x; alive && (!WALK || item < n_items); item += gridDim.x) {
-      Item it = it0;
-      if (WALK && !decode(item, it)) continue;
+    while (alive) {
+      const uint32_t slot = n & 1;
+      const bool published = mbar_wait(&item_full[slot], (n >> 1) & 1, abort_flag);
+      if (!__all_sync(0xffffffffu, published)) break;
+      const int item = item_slot[slot];
+      __syncwarp();                                     // every lane has read the slot
+      if (lane == 0) mbar_arrive(&item_empty[slot]);
+      ++n;
+      if (item < 0) break;
+      Item it;
+      if (!decode(item, it)) continue;
       const int h = it.h, b = it.b, nq = it.nq, s_first = it.s_first;
-      for (int pass = 0; alive && pass < N_PASS; ++pass) {
-        if (pass == 1) {
-          const bool known = mbar_wait(verdict, 0, abort_flag);
-          if (!__all_sync(0xffffffffu, known)) { alive = false; break; }
-          if (!*redo) break;
-        }
-        const bool safe = pass == 1;                      // running maximum on every tile
-        float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
-        for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
-          const uint32_t buf = kc & 1;
-          const int j0 = (kt_lo + kt) * BK;
-          const bool landed = mbar_wait(&s_full[buf], (kc >> 1) & 1, abort_flag);
-          if (!__all_sync(0xffffffffu, landed)) { alive = false; break; }   // the TMEM loads below are warp-wide
-          tc_fence_after();
-          float v[NC][32];
-#pragma unroll
-          for (int c = 0; c < NC; ++c) tmem_ld32(lane_addr + buf * BK + c * 32, v[c]);
+      float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
+      for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
+        const uint32_t buf = kc % XT_SBUF;
+        const bool landed = mbar_wait(&s_full[buf], (kc / XT_SBUF) & 1, abort_flag);
+        if (!__all_sync(0xffffffffu, landed)) { alive = false; break; }   // the TMEM loads below are warp-wide
+        tc_fence_after();
+        const int n_half = min(2, it.nsub - 2 * kt);     // halves of this tile the item needs
+        for (int half = 0; half < n_half; ++half) {
+          const int j0 = (kt_lo + kt) * BK + half * XT_SUB + cg * 32;      // first key of this thread's 32 columns
+          float v[32];
+          tmem_ld32(lane_addr + buf * BK + half * XT_SUB, v);
           tmem_ld_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&s_empty[buf]);
+          if (half == n_half - 1) {                       // the accumulator is in registers: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_empty[buf]);
+          }
 
-          if (WALK) {                                       // normaliser known: only the prompt columns count
+          if (LSE) {                                      // normaliser known: only the prompt columns count
             const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
-            const unsigned long long tm = a.text.mask64(j0);
+            const unsigned int tm = (unsigned int)a.text.mask64(j0);
             float st = 0.f;
 #pragma unroll
-            for (int c = 0; c < NC; ++c)
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if ((tm >> (c * 32 + i)) & 1ull) st += ex2(fmaf(v[c][i], sc, -l2));
+            for (int i = 0; i < 32; ++i)
+              if ((tm >> i) & 1u) st += ex2(fmaf(v[i], sc, -l2));
             l_txt += st;
             l_all = 1.f;
             continue;
           }
-          const bool in_j = j0 < a.text.end && j0 + BK > a.text.begin;   // tile reaches into the prompt set J
-          // some row of the tile does not see all of its keys: the diagonal, or the end of the sample
-          const bool edge = j0 + BK - 1 > (a.bidirectional ? it.n_seq - 1 : s_first);
-          int lim_max = BK;                                // columns at least one row of this warp sees
+          const bool in_j = j0 < a.text.end && j0 + 32 > a.text.begin;     // the columns reach into the prompt set J
+          // some row does not see all of these keys: the diagonal, or the end of the sample
+          const bool edge = j0 + 31 > (a.bidirectional ? it.n_seq - 1 : s_first);
+          int lim_max = 32;                                // columns at least one row of this warp sees
           if (edge) {
             const int lim = (a.bidirectional ? it.n_seq - 1 : s_first + r) - j0;   // last visible column of this row
             lim_max = __reduce_max_sync(0xffffffffu, lim);
-            if (lim_max < 0) continue;                     // no row of this warp sees any key of the tile
+            if (lim_max < 0) continue;                     // no row of this warp sees any of these keys
 #pragma unroll
-            for (int c = 0; c < NC; ++c)
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (c * 32 + i > lim) v[c][i] = -INFINITY;
+            for (int i = 0; i < 32; ++i)
+              if (i > lim) v[i] = -INFINITY;
           }
-          if (kt == 0 || safe) {
-            // reference of the row: maximum of the first tile (every row sees key 0), of every tile when safe
+          if (SAFE || __any_sync(0xffffffffu, m_run == -INFINITY)) {
+            // reference of the thread: maximum of the first 32 columns of its own in which it sees a key (the
+            // first 64 keys of the row, unless the row is among the first 32 of a sequence), of every half when
+            // SAFE.  While some row of the warp has no reference yet the others update theirs, which is exact.
             float mx[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              mx[j] = v[j / 2][(j & 1) * 16];
+              mx[j] = v[j * 8];
 #pragma unroll
-              for (int i = 1; i < 16; ++i) mx[j] = fmaxf(mx[j], v[j / 2][(j & 1) * 16 + i]);
+              for (int i = 1; i < 8; ++i) mx[j] = fmaxf(mx[j], v[j * 8 + i]);
             }
             const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), m_run);
-            const float resc = ex2((m_run - m_new) * sc);     // 0 on the first tile
-            l_all *= resc;
-            l_txt *= resc;
-            m_run = m_new;
+            if (m_new > -INFINITY) {                        // (a thread whose 32 columns are all masked keeps none)
+              const float resc = ex2((m_run - m_new) * sc); // 0 on the first half
+              l_all *= resc;
+              l_txt *= resc;
+              m_run = m_new;
+            }
           }
+          if (m_run == -INFINITY) continue;                // this thread has not seen a key yet
           const float ms = m_run * sc;
           if (!edge && !in_j) {
-            // the bulk of the tiles: every fourth exponential on the FMA pipe
+            // the bulk: every fourth exponential on the FMA pipe
             float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < NC; ++c)
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const float x = fmaf(v[c][i], sc, -ms);
-                part[(i & 1) + 2 * c] += (i & 3) == 3 ? ex2_fma(x) : ex2(x);
-              }
+            for (int i = 0; i < 32; ++i) {
+              const float x = fmaf(v[i], sc, -ms);
+              part[i & 3] += (i & 3) == 3 ? ex2_fma(x) : ex2(x);
+            }
             l_all += (part[0] + part[1]) + (part[2] + part[3]);
           } else {
-            const unsigned long long tm = in_j ? a.text.mask64(j0) : 0ull;
+            const unsigned int tm = in_j ? (unsigned int)a.text.mask64(j0) : 0u;
             float sa = 0.f, st = 0.f;
 #pragma unroll
-            for (int c = 0; c < NC; ++c)
+            for (int blk = 0; blk < 4; ++blk)
+              if (blk * 8 <= lim_max) {                     // warp-uniform: masked blocks cost no exponentials
+                float pa = 0.f, pt = 0.f;
 #pragma unroll
-              for (int blk = 0; blk < 4; ++blk)
-                if (c * 32 + blk * 8 <= lim_max) {          // warp-uniform: masked blocks cost no exponentials
-                  float pa = 0.f, pt = 0.f;
-#pragma unroll
-                  for (int i = 0; i < 8; ++i) {
-                    const float p = ex2(fmaf(v[c][blk * 8 + i], sc, -ms));   // exp2(-inf) = 0 on masked columns
-                    pa += p;
-                    if ((tm >> (c * 32 + blk * 8 + i)) & 1ull) pt += p;
-                  }
-                  sa += pa;
-                  st += pt;
+                for (int i = 0; i < 8; ++i) {
+                  const float p = ex2(fmaf(v[blk * 8 + i], sc, -ms));   // exp2(-inf) = 0 on masked columns
+                  pa += p;
+                  if ((tm >> (blk * 8 + i)) & 1u) pt += p;
                 }
+                sa += pa;
+                st += pt;
+              }
             l_all += sa;
             l_txt += st;
           }
-        }
+        }  // halves
+      }  // key tiles
+      // ---- the two threads of a row meet: the upper column group hands its reference and sums over.  Every warp
+      //      that entered the item takes part, also after a failed wait (the flag is raised, nothing is stored).
+      if (cg == 1) {
+        const bool free_again = np == 0 || mbar_wait(pair_empty, (np - 1) & 1, abort_flag);
+        if (!__all_sync(0xffffffffu, free_again)) alive = false;
+        pair_m[r] = m_run; pair_all[r] = l_all; pair_txt[r] = l_txt;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pair_full);
+        ++np;
         if (!alive) break;
-        if (!WALK && pass == 0) {
-          // a sum that is not a finite positive number means some logit lay more than 88 above the reference
-          const bool bad = r < nq && !(l_all <= 3.0e38f);
-          const bool any_bad = __any_sync(0xffffffffu, bad);
-          if (lane == 0) {
-            if (any_bad) atomicOr(redo, 1);
-            mbar_arrive(verdict);
-          }
-        }
-        if (r < nq && !*abort_flag) {
-          a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + it.t0 + r] = WALK ? l_txt : l_txt / l_all;
-          if (!WALK && a.lse_out)
-            a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + s_first + r] =
-                fmaf(m_run, sc, log2f(l_all)) * 0.6931471805599453f;
-        }
+        continue;
       }
-      if (!WALK) break;
+      {
+        const bool handed = mbar_wait(pair_full, np & 1, abort_flag);
+        if (!__all_sync(0xffffffffu, handed)) alive = false;
+        ++np;
+        if (!alive) break;
+        if (!LSE) {
+          const float m_o = pair_m[r], m_new = fmaxf(m_run, m_o);
+          const float f_own = ex2((m_run - m_new) * sc), f_o = m_o > -INFINITY ? ex2((m_o - m_new) * sc) : 0.f;
+          l_all = fmaf(l_all, f_own, pair_all[r] * f_o);
+          l_txt = fmaf(l_txt, f_own, pair_txt[r] * f_o);
+          m_run = m_new;
+        } else {
+          l_txt += pair_txt[r];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pair_empty);             // the exchange buffers are free for the next item
+      }
+      if (!LSE && !SAFE) {
+        // a sum that is not a finite number means some logit lay more than 88 above the reference: the item
+        // goes on the list of the second launch (once per CTA)
+        const bool bad = r < nq && !(l_all <= 3.0e38f);
+        if (__any_sync(0xffffffffu, bad) && lane == 0 && atomicExch(redo_mark, item) != item)
+          a.redo_list[atomicAdd(&a.sched->n_redo, 1u)] = item;
+      }
+      if (r < nq && !*abort_flag) {
+        a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + it.t0 + r] = LSE ? l_txt : l_txt / l_all;
+        if (!LSE && a.lse_out)
+          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + s_first + r] =
+              fmaf(m_run, sc, log2f(l_all)) * 0.6931471805599453f;
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 2 * BK);
+    tmem_dealloc(tmem_base, XT_SBUF * BK);
   }
   if (threadIdx.x == 0 && *abort_flag && a.status) atomicOr(a.status, LIGHTKV_STATUS_TIMEOUT);
 }
@@ -404,24 +476,27 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   x.n_q_heads = L.n_q_heads; x.group = L.n_q_heads / L.n_kv_heads;
   x.scale2 = 1.4426950408889634f / sqrtf((float)L.head_dim);
   x.batch = L.batch; x.n_qt = (L.ws.cap_in + 127) / 128;
-  // One CTA per work item when the rows are long (the hardware balances them, and kernels on other streams
-  // find room as CTAs retire).  With the caller's log-sum-exp an item is two or three key tiles, all items
-  // alike: then as many CTAs as stay resident (three per SM) walk the list, and the next item's loads hide
-  // behind the current one's arithmetic.
-  const bool walk = x.lse != nullptr;
+  x.sched = reinterpret_cast<XiSched*>(L.ws.xi_sched); x.redo_list = L.ws.xi_redo;
   const long long n_items = (long long)x.n_qt * L.n_q_heads * L.batch;
   if (n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
-  const dim3 grid = walk ? dim3((unsigned)std::min<long long>(n_items, (XT_KEY_TILE == 64 ? 3 : 2) * sm_count()))
-                         : dim3(x.n_qt, L.n_q_heads, L.batch);
-  constexpr int BK = XT_KEY_TILE;
-  const size_t smem = size_t(L.head_dim / 64) * (16384 + size_t(XT_STAGES) * BK * 128) + 1024 + 256;
-  auto launch = [&](auto kernel) -> cudaError_t {
-    const cudaError_t e = ensure_dynamic_smem(kernel, (int)smem);
-    if (e != cudaSuccess) return e;
-    return launch_kernel(kernel, grid, 192, smem, L.stream, 1, qm, km, x);
+  // As many CTAs as stay resident (two per SM) draw work items from a ticket counter; with the caller's
+  // log-sum-exp an item is one or two key tiles, otherwise up to the whole row.
+  const dim3 grid((unsigned)std::min<long long>(n_items, XT_CTAS * sm_count()));
+  const size_t smem = size_t(L.head_dim / 64) * (16384 + size_t(XT_STAGES) * XT_KEY_TILE * 128) + 1024 + 256 + 1536;
+  cudaError_t e = cudaMemsetAsync(x.sched, 0, sizeof(XiSched), L.stream);      // tickets and list length start at 0
+  if (e != cudaSuccess) return e;
+  auto launch = [&](auto kernel, dim3 g) -> cudaError_t {
+    const cudaError_t rc = ensure_dynamic_smem(kernel, (int)smem);
+    if (rc != cudaSuccess) return rc;
+    return launch_kernel(kernel, g, XT_THREADS, smem, L.stream, 1, qm, km, x);
   };
-  if (L.head_dim == 128) return walk ? launch(xi_tc_kernel<128, BK, true>) : launch(xi_tc_kernel<128, BK, false>);
-  return walk ? launch(xi_tc_kernel<64, BK, true>) : launch(xi_tc_kernel<64, BK, false>);
+  if (x.lse) return L.head_dim == 128 ? launch(xi_tc_kernel<128, true, false>, grid) : launch(xi_tc_kernel<64, true, false>, grid);
+  e = L.head_dim == 128 ? launch(xi_tc_kernel<128, false, false>, grid) : launch(xi_tc_kernel<64, false, false>, grid);
+  if (e != cudaSuccess) return e;
+  // second launch: the items whose sums left the fp32 range, with a running maximum (returns at once when the
+  // list is empty; one CTA per SM is plenty for what is an exception)
+  const dim3 grid2((unsigned)std::min<long long>(n_items, sm_count()));
+  return L.head_dim == 128 ? launch(xi_tc_kernel<128, false, true>, grid2) : launch(xi_tc_kernel<64, false, true>, grid2);
 }
 
 // ======================================================================================================
