@@ -197,6 +197,11 @@ def build_inputs(wl, plan, L, torch, device, sample_offset, kv_layout="bhnd", xi
 
 
 def run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None, side=None, aux=None):
+    k_dst, v_dst = (stg["dev"]["k"], stg["dev"]["v"]) if stg.get("kv_in_place") else (stg["k_dst"], stg["v_dst"])
+    return _run_stage(L, plan, wl, st, stg, pos, n_vis, trace, side, aux, k_dst, v_dst)
+
+
+def _run_stage(L, plan, wl, st, stg, pos, n_vis, trace, side, aux, k_dst, v_dst):
     """lightkv_compress_layer on the current stream, then lightkv_compact_kv either on the same stream or,
     when `side` is given, on that stream behind the call's map event (the compaction only needs the stage's
     merge map, which is complete before the hidden-state merge starts)."""
@@ -206,15 +211,14 @@ def run_stage(L, plan, wl, st, stg, pos, n_vis, trace=None, side=None, aux=None)
     L.compress_layer(plan, st, d["hidden"], stg["out"], vis_begin=wl.n_text, q=d["q"], k=d["k"], n_vis=n_vis,
                      pos=pos, trace_events=trace, aux_stream=aux, lse=d.get("lse"), map_event=map_event)
     if side is None:
-        L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
-                     n_vis=n_vis)
+        L.compact_kv(plan, st, stg["out"], d["k"], d["v"], k_dst, v_dst, vis_begin=wl.n_text, n_vis=n_vis)
     else:
         if map_event is not None:
             side.wait_event(map_event)
         else:
             side.wait_stream(torch.cuda.current_stream())
-        L.compact_kv(plan, st, stg["out"], d["k"], d["v"], stg["k_dst"], stg["v_dst"], vis_begin=wl.n_text,
-                     n_vis=n_vis, stream=side)
+        L.compact_kv(plan, st, stg["out"], d["k"], d["v"], k_dst, v_dst, vis_begin=wl.n_text, n_vis=n_vis,
+                     stream=side)
 
 
 def run_step(L, plan, wl, stages, traces=None, kv_events=None, side=None, aux=None):
@@ -325,6 +329,8 @@ def main():
                          "is an input (computed once with torch before the timed region), only prompt keys are visited")
     ap.add_argument("--kv-layout", default="bhnd", choices=["bhnd", "bnhd"],
                     help="K/V cache layout: [B,H_kv,N,dh] (head-major) or [B,N,H_kv,dh] (token-major)")
+    ap.add_argument("--kv-in-place", action="store_true",
+                    help="compact K/V inside the cache's own rows (destination = source) instead of into a second buffer")
     ap.add_argument("--graph", type=int, default=1, choices=[0, 1],
                     help="1: replay the step from a CUDA graph captured once (timed region only)")
     ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
@@ -343,7 +349,7 @@ def main():
                           f"keep={list(wl.keep)}, batch {wl.batch}, {wl.n_vis} vision + {wl.n_text} text tokens, "
                           f"hidden {wl.hidden}, {wl.n_q_heads}q/{wl.n_kv_heads}kv heads x {wl.head_dim}, "
                           f"xi from {'full causal attention' if args.xi_mode == 'full' else 'the prompt keys + a given row log-sum-exp'}, "
-                          f"K/V merge, K/V layout {args.kv_layout}",
+                          f"K/V merge{' in place' if args.kv_in_place else ''}, K/V layout {args.kv_layout}",
               "batch_per_gpu": wl.batch}
     # L2 policy of the device-timed arm, a function of the workload alone so that both arms print the same config:
     # a step streams every stage's inputs once; where the first stage's inputs are less than twice the L2, the L2
@@ -402,6 +408,8 @@ def main():
                   engine=L.ENGINE_AUTO if args.engine == "auto" else L.ENGINE_SIMT)
     stages = build_inputs(wl, plan, L, torch, device, sample_offset=rank * wl.batch, kv_layout=args.kv_layout,
                           xi_mode=args.xi_mode)
+    for s in stages:
+        s["kv_in_place"] = args.kv_in_place
     tokens_per_step = int(sum(int(s["n_vis"].sum()) for s in stages))
     n_stages = len(stages)
 

@@ -265,12 +265,20 @@ int lightkv_compress_layer(const lightkv_plan_t* plan, const lightkv_layer_args_
 #define LIGHTKV_BUILTIN_WS_BYTES (8u << 20)
 int lightkv_compress_layer_builtin_ws(const lightkv_plan_t* plan, const lightkv_layer_args_t* args);
 
-/* Apply a stage's merge map to one layer's K and V (out of place).
+/* Apply a stage's merge map to one layer's K and V.
  * Contiguous: element (b, h, n, :) of a tensor lives at
  *   base + b*batch_stride + h*head_stride + n*row_stride.
  * Paged (page_size > 0): token n of sample b lives in page block_table[b*max_blocks + n/page_size] at
  *   base + page*page_stride + h*head_stride + (n % page_size)*row_stride.
- * Text rows are copied; vision rows are merged or gathered per `mode`. */
+ * Text rows are copied; vision rows are merged or gathered per `mode`.
+ * Out of place: the destinations do not overlap the sources.
+ * In place: k_dst == k_src and v_dst == v_src with the same strides, page size and block table on both sides
+ * (anything else that overlaps is INVALID_ARG or undefined).  The cache then shrinks inside its own rows or
+ * pages, with no second copy of it: first every merged group is written over its surviving token's row (no
+ * other group reads that row), then every output row moves forward to its slot -- a slot never lies behind its
+ * source -- one (sample, K or V, head) plane per CTA, in ascending chunks that are gathered into shared memory
+ * before any of their slots is written.  Rows behind the new end of a sample keep stale contents; pages that
+ * became empty are the caller's to release. */
 typedef struct {
   uint32_t struct_size;            /* sizeof(lightkv_kv_args_t) */
   int32_t  stage;
@@ -282,7 +290,7 @@ typedef struct {
   const int32_t* grp_src;
   const float*   weight;
   const void* k_src; const void* v_src;      /* DEVICE */
-  void* k_dst; void* v_dst;                  /* DEVICE; must not overlap the sources */
+  void* k_dst; void* v_dst;                  /* DEVICE; disjoint from the sources, or equal to them (in place) */
   int64_t src_batch_stride, src_head_stride, src_row_stride;
   int64_t dst_batch_stride, dst_head_stride, dst_row_stride;
   int32_t page_size;               /* 0 = contiguous */

@@ -867,7 +867,7 @@ template <typename T>
 __global__ void __launch_bounds__(KV_THREADS, sizeof(T) == 2 ? 5 : 4)
 kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* __restrict__ k_dst,
                   T* __restrict__ v_dst, KvAddr sa, KvAddr da, int n_kv_heads, int dh, int vis_begin,
-                  int n_text_after, int cap_in, int cap_out, int gather, unsigned magic_ch,
+                  int n_text_after, int cap_in, int cap_out, int gather, int merge_at_survivor, unsigned magic_ch,
                   const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
                   const int* __restrict__ grp_off, const int* __restrict__ grp_src,
                   const float* __restrict__ weight) {
@@ -878,7 +878,7 @@ kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* _
   const int n_out = n_vis_out[b];
   if (row >= vis_begin + n_out + n_text_after) return;
   const int ch = dh / V, per_kv = n_kv_heads * ch, units = 2 * per_kv;
-  const int64_t d_tok = da.token(b, row);
+  int64_t d_tok = da.token(b, row);
   const bool text = row < vis_begin || row >= vis_begin + n_out;
   const int* gs = grp_src + size_t(b) * cap_in;
   const float* wt = weight + size_t(b) * cap_in;
@@ -887,6 +887,12 @@ kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* _
     const int* go = grp_off + size_t(b) * (cap_out + 1);
     g0 = go[row - vis_begin];
     g1 = gather ? g0 + 1 : go[row - vis_begin + 1];
+  }
+  if (merge_at_survivor) {
+    // first phase of the in-place form: a merged group is written over its surviving token's own row (no other
+    // group reads that row); rows that are only moved wait for the second phase
+    if (text || g1 - g0 == 1) return;
+    d_tok = da.token(b, vis_begin + gs[g0]);
   }
   if (text || g1 - g0 == 1) {                                       // copy: text, lone survivor, gather mode
     const int64_t s_tok = text ? sa.token(b, row < vis_begin ? row : row - n_out + n_in)
@@ -957,6 +963,71 @@ kv_compact_kernel(const T* __restrict__ k_src, const T* __restrict__ v_src, T* _
   }
 }
 
+// =====================================================================================================
+// Second phase of the in-place form: every output row moves from its surviving token's row (which holds the
+// merged group after the first phase) to its slot.  A slot never lies behind its source (o <= i), so rows only
+// move towards the front.  One CTA owns a plane -- one (sample, K or V, head, column part) -- and sweeps its
+// output rows in ascending chunks: the sources of a chunk are gathered into shared memory, the CTA
+// synchronises, the chunk is stored.  The sources of chunk k + 1 lie at or behind its first slot, i.e. behind
+// everything chunk k writes, so its gather is issued before chunk k is stored; and a chunk's own sources are in
+// shared memory before any of its slots is written.  Rows before the vision block do not move.
+// =====================================================================================================
+constexpr int KVM_THREADS = 256, KVM_CHUNK_BYTES = 40 * 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(KVM_THREADS)
+kv_move_kernel(T* __restrict__ k_buf, T* __restrict__ v_buf, KvAddr ad, int n_kv_heads, int dh, int parts,
+               int vis_begin, int n_text_after, int cap_in, const int* __restrict__ n_vis,
+               const int* __restrict__ n_vis_out, const int* __restrict__ grp_off, const int* __restrict__ grp_src,
+               int cap_out) {
+  grid_dependency_sync();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int V = Vec<T>::n;
+  int plane = blockIdx.x;
+  const int part = plane % parts; plane /= parts;
+  const int h = plane % n_kv_heads; plane /= n_kv_heads;
+  const int kv = plane & 1, b = plane >> 1;
+  const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
+  const int n_out = n_vis_out[b];
+  if (n_out >= n_in) return;                               // nothing was merged away: every row is where it belongs
+  T* buf = (kv ? v_buf : k_buf) + int64_t(h) * ad.head_stride;
+  const int ch_all = dh / V, ch0 = part * ch_all / parts, ch = (part + 1) * ch_all / parts - ch0;   // 16-byte pieces of this plane
+  const int rows_per_chunk = KVM_CHUNK_BYTES / (ch * 16);
+  const int* go = grp_off + size_t(b) * (cap_out + 1);
+  const int* gs = grp_src + size_t(b) * cap_in;
+  const int row_end = vis_begin + n_out + n_text_after;
+  const uint32_t sbase = tc::smem_u32(smem_raw);
+  auto source = [&](int row) {                            // row of the buffer that holds output row `row`
+    return row < vis_begin + n_out ? vis_begin + gs[go[row - vis_begin]] : row - n_out + n_in;
+  };
+  auto gather = [&](int r0, uint32_t sm) {                // output rows r0 .. of one chunk -> shared memory
+    const int nr = min(rows_per_chunk, row_end - r0);
+    for (int idx = threadIdx.x; idx < nr * ch; idx += blockDim.x) {
+      const int rr = idx / ch, c = idx - rr * ch;
+      tc::cp_async16(sm + uint32_t(idx) * 16, buf + ad.token(b, source(r0 + rr)) + (ch0 + c) * V, 16);
+    }
+  };
+  int r0 = vis_begin, k = 0;
+  gather(r0, sbase);
+  tc::cp_async_commit();
+  for (; r0 < row_end; r0 += rows_per_chunk, ++k) {
+    const int next = r0 + rows_per_chunk;
+    if (next < row_end) gather(next, sbase + ((k + 1) & 1) * KVM_CHUNK_BYTES);
+    tc::cp_async_commit();
+    tc::cp_async_wait<1>();                               // this thread's pieces of chunk k have landed
+    __syncthreads();                                      // ... and everybody else's: all sources of chunk k are on chip
+    const int nr = min(rows_per_chunk, row_end - r0);
+    const unsigned char* sm = smem_raw + (k & 1) * KVM_CHUNK_BYTES;
+    for (int idx = threadIdx.x; idx < nr * ch; idx += blockDim.x) {
+      const int rr = idx / ch, c = idx - rr * ch;
+      const uint4 v = *reinterpret_cast<const uint4*>(sm + size_t(idx) * 16);
+      st_stream16(buf + ad.token(b, r0 + rr) + (ch0 + c) * V, v);
+    }
+    __syncthreads();                                      // the buffer may be refilled two chunks on
+  }
+  tc::cp_async_wait<0>();
+}
+
 cudaError_t launch_kv_compact(const KvLaunch& K) {
   const lightkv_kv_args_t* a = K.a;
   KvAddr sa{a->src_batch_stride, a->src_head_stride, a->src_row_stride, a->src_page_stride,
@@ -971,17 +1042,26 @@ cudaError_t launch_kv_compact(const KvLaunch& K) {
   // two units per thread (both in flight); narrow caches (GQA) get narrow CTAs
   const int threads = std::min(KV_THREADS, ((units + 1) / 2 + 31) / 32 * 32);
   const int gather = a->mode == LIGHTKV_KV_GATHER;
-  if (K.dtype == LIGHTKV_BF16)
-    return launch_kernel(kv_compact_kernel<__nv_bfloat16>, grid, threads, 0, K.stream, 1,
-        static_cast<const __nv_bfloat16*>(a->k_src), static_cast<const __nv_bfloat16*>(a->v_src),
-        static_cast<__nv_bfloat16*>(a->k_dst), static_cast<__nv_bfloat16*>(a->v_dst), sa, da, K.n_kv_heads,
-        K.head_dim, a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, magic_ch, a->n_vis,
-        a->n_vis_out, a->grp_off, a->grp_src, a->weight);
-  return launch_kernel(kv_compact_kernel<float>, grid, threads, 0, K.stream, 1,
-        static_cast<const float*>(a->k_src), static_cast<const float*>(a->v_src),
-        static_cast<float*>(a->k_dst), static_cast<float*>(a->v_dst), sa, da, K.n_kv_heads, K.head_dim,
-        a->vis_begin, a->n_text_after, K.cap_in, K.cap_out, gather, magic_ch, a->n_vis, a->n_vis_out,
-        a->grp_off, a->grp_src, a->weight);
+  const bool in_place = a->k_src == a->k_dst;             // (the API checked that V and the addressing agree)
+  auto run = [&](auto tag) -> cudaError_t {
+    using T = decltype(tag);
+    cudaError_t e = cudaSuccess;
+    if (!(in_place && gather))                            // in place, gather mode has nothing to merge
+      e = launch_kernel(kv_compact_kernel<T>, grid, threads, 0, K.stream, 1,
+          static_cast<const T*>(a->k_src), static_cast<const T*>(a->v_src), static_cast<T*>(a->k_dst),
+          static_cast<T*>(a->v_dst), sa, da, K.n_kv_heads, K.head_dim, a->vis_begin, a->n_text_after, K.cap_in,
+          K.cap_out, gather, in_place ? 1 : 0, magic_ch, a->n_vis, a->n_vis_out, a->grp_off, a->grp_src, a->weight);
+    if (e != cudaSuccess || !in_place) return e;
+    // planes: (sample, K / V, head), cut along head_dim while there are fewer of them than CTAs that fit
+    int parts = 1;
+    while (parts < ch_host && K.batch * 2 * K.n_kv_heads * parts < 4 * 148 && ch_host % (2 * parts) == 0) parts *= 2;
+    const size_t smem = 2 * size_t(KVM_CHUNK_BYTES);
+    if ((e = ensure_dynamic_smem(kv_move_kernel<T>, (int)smem)) != cudaSuccess) return e;
+    return launch_kernel(kv_move_kernel<T>, dim3(K.batch * 2 * K.n_kv_heads * parts), KVM_THREADS, smem, K.stream, 1,
+        static_cast<T*>(a->k_dst), static_cast<T*>(a->v_dst), da, K.n_kv_heads, K.head_dim, parts, a->vis_begin,
+        a->n_text_after, K.cap_in, a->n_vis, a->n_vis_out, a->grp_off, a->grp_src, K.cap_out);
+  };
+  return K.dtype == LIGHTKV_BF16 ? run(__nv_bfloat16()) : run(float());
 }
 
 }  // namespace lkv

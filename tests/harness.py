@@ -103,7 +103,8 @@ def make_plan(wl, dtype="bf16", xi_mode="attn", engine="auto", batch=None, max_t
 
 def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0, text_range=None,
               lse=None, kv_mode="merge", paged=0, device="cuda", layer_fn=None, aux_stream=None,
-              kv_layout="bhnd", kv_stream=None, text_ranges=None, bidirectional=False, want_lse=False):
+              kv_layout="bhnd", kv_stream=None, text_ranges=None, bidirectional=False, want_lse=False,
+              kv_in_place=False):
     """Run lightkv_compress_layer (or `layer_fn`, a binding function with the same signature) +
     lightkv_compact_kv on the device; returns numpy outputs."""
     import torch
@@ -177,9 +178,13 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
                     lo, hi = blk * paged, min(n_seq, (blk + 1) * paged)
                     ks[perm_s[b, blk], :, :hi - lo] = k_src[b, :, lo:hi]
                     vs[perm_s[b, blk], :, :hi - lo] = v_src[b, :, lo:hi]
+            if kv_in_place:     # the page pool shrinks inside its own pages: one pool, one block table
+                kd, vd, perm_d = ks, vs, perm_s
+            table_s = perm_s.to(device)
+            table_d = table_s if kv_in_place else perm_d.to(device)
             L.compact_kv(plan, stage, out, ks, vs, kd, vd, vis_begin=vb, n_text_after=n_text_after, mode=mode,
                          n_vis=torch.from_numpy(inp["n_vis"]).to(device), page_size=paged,
-                         src_block_table=perm_s.to(device), dst_block_table=perm_d.to(device))
+                         src_block_table=table_s, dst_block_table=table_d)
             torch.cuda.synchronize()
             k_dst = torch.full((bsz, hkv, n_seq_out, dh), float("nan"), dtype=tdt, device=device)
             v_dst = k_dst.clone()
@@ -195,8 +200,12 @@ def gpu_stage(plan, wl, stage, inp, dtype="bf16", xi_mode="attn", n_text_after=0
                 as_bnhd = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
                 k_src, v_src, k_dst, v_dst = as_bnhd(k_src), as_bnhd(v_src), as_bnhd(k_dst), as_bnhd(v_dst)
                 assert k_src.stride(1) == dh and k_src.stride(2) == hkv * dh
+            if kv_in_place:     # destination = source (the shorter sequences end up at the front of their rows)
+                k_dst, v_dst = k_src, v_src
             L.compact_kv(plan, stage, out, k_src, v_src, k_dst, v_dst, vis_begin=vb, n_text_after=n_text_after,
                          mode=mode, n_vis=torch.from_numpy(inp["n_vis"]).to(device), **kv_kw)
+            if kv_in_place:
+                k_dst, v_dst = k_dst[:, :, :n_seq_out], v_dst[:, :, :n_seq_out]
         torch.cuda.synchronize()
         res["k_out"], res["v_out"] = k_dst.float().cpu().numpy(), v_dst.float().cpu().numpy()
     torch.cuda.synchronize()
@@ -283,7 +292,7 @@ def check_lse_out(inp, gpu, n_heads, n_kv, samples, causal=True, n_text_after=0,
 def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge", paged=0, samples=None,
                  stages=None, oracle_samples=None, aux_stream=None, kv_layout="bhnd", kv_stream=None,
                  lse_source="oracle", ragged=False, first_pos=None, text_ranges=None, bidirectional=False,
-                 want_lse=False, expect_status=0, metric="cosine", direction="a2b"):
+                 want_lse=False, expect_status=0, metric="cosine", direction="a2b", kv_in_place=False):
     """All stages of a workload, chained through the surviving positions; returns per-stage stats.
     first_pos: per-sample positions entering stage 0 (a subset of the grid); ragged: plan built for subsets."""
     bsz = wl.batch if samples is None else len(samples)
@@ -301,7 +310,7 @@ def run_schedule(wl, dtype="bf16", xi_mode="attn", engine="auto", kv_mode="merge
                                                                    causal=not bidirectional)
         gpu = gpu_stage(plan, wl, stage, inp, dtype, xi_mode, lse=lse, kv_mode=kv_mode, paged=paged,
                         aux_stream=aux_stream, kv_layout=kv_layout, kv_stream=kv_stream, text_ranges=text_ranges,
-                        bidirectional=bidirectional, want_lse=want_lse)
+                        bidirectional=bidirectional, want_lse=want_lse, kv_in_place=kv_in_place)
         osamp = list(range(bsz)) if oracle_samples is None else oracle_samples
         sub = {key: (val[osamp] if isinstance(val, np.ndarray) and val.shape[:1] == (bsz,) else val)
                for key, val in inp.items()}

@@ -200,9 +200,13 @@ def test_calls_reject_bad_arguments_before_any_launch(L):
     kv.mode = 0
     for f in ("n_vis_out", "grp_off", "grp_src", "weight", "k_src", "v_src"):
         setattr(kv, f, 0x1000)
-    kv.k_dst = kv.v_dst = 0x1000
+    kv.k_dst, kv.v_dst = 0x1000, 0x3000
     kv.src_row_stride = kv.dst_row_stride = 16
-    assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1               # in place is not supported
+    assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1               # K in place, V not
+    kv.k_dst = kv.v_dst = 0x1000
+    kv.dst_head_stride = 16 * 64
+    assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1               # in place with two addressings
+    kv.dst_head_stride = 0
     kv.k_dst = kv.v_dst = 0x3000
     kv.page_size = 16
     assert lib.lightkv_compact_kv(p.handle, C.byref(kv)) == -1               # paged without block tables

@@ -252,6 +252,49 @@ def test_logits_far_above_the_first_tiles_maximum_take_the_safe_pass(name):
     plan.close()
 
 
+# ---- K/V compaction inside the cache's own rows / pages ---------------------------------------------------------
+
+@pytest.mark.parametrize("kv_mode,paged,layout", [("merge", 0, "bhnd"), ("gather", 0, "bhnd"), ("merge", 16, "bhnd"),
+                                                  ("merge", 5, "bhnd"), ("gather", 16, "bhnd"), ("merge", 0, "bnhd")])
+def test_in_place_kv_compaction(kv_mode, paged, layout):
+    # destination = source: groups are merged over their surviving token's row, then rows move forward plane by
+    # plane; compared with the oracle like the out-of-place form (ragged windows, two tiles, GQA, three stages)
+    H.run_schedule(S.workload("small"), kv_mode=kv_mode, paged=paged, kv_layout=layout, kv_in_place=True)
+
+
+def test_in_place_kv_compaction_long_rows_and_text_behind():
+    # 2304 tokens per sample: a plane is swept in many chunks (sources of a chunk lie inside the next chunks'
+    # destinations); text rows behind the vision block move forward with it
+    wl = S.Workload(name="inpl", config_id=140, batch=2, tiles=((48, 48),), n_text=37, hidden=64, n_q_heads=4,
+                    n_kv_heads=2, head_dim=64, n_layers=16, layers=(3, 7), windows=(6, 3), keep=(0.55, 0.5))
+    H.run_schedule(wl, xi_mode="given", kv_in_place=True)
+    plan = H.make_plan(wl, xi_mode="uniform")
+    inp = H.prepare_stage(wl, 0)
+    vb, after = wl.n_text - 9, 9
+    for key in ("hidden", "q", "k", "v"):
+        a = inp[key]
+        axis = 1 if key == "hidden" else 2
+        a = np.concatenate([np.take(a, range(0, vb), axis), np.take(a, range(wl.n_text, a.shape[axis]), axis),
+                            np.take(a, range(vb, wl.n_text), axis)], axis)
+        inp[key] = np.ascontiguousarray(a)
+    inp["vis_begin"] = vb
+    gpu = H.gpu_stage(plan, wl, 0, inp, xi_mode="uniform", n_text_after=after, kv_in_place=True)
+    ref = H.oracle_stage(wl, 0, inp, "uniform", n_text_after=after)
+    H.compare_stage(wl, 0, inp, ref, gpu, n_text_after=after)
+    plan.close()
+
+
+def test_in_place_equals_out_of_place_bit_for_bit():
+    wl = S.workload("cfg1")
+    plan = H.make_plan(wl)
+    inp = H.prepare_stage(wl, 0, repair=False)
+    a = H.gpu_stage(plan, wl, 0, inp)
+    b = H.gpu_stage(plan, wl, 0, inp, kv_in_place=True)
+    np.testing.assert_array_equal(a["k_out"], b["k_out"])
+    np.testing.assert_array_equal(a["v_out"], b["v_out"])
+    plan.close()
+
+
 # ---- the variants the paper ablates: Euclidean pair scores, reverse message direction ---------------------------
 
 @pytest.mark.parametrize("metric", ["l2sq", "l2"])
