@@ -233,6 +233,13 @@ typedef struct {
                                       check its fused attention's own, or feed a later call.  Rows outside
                                       the vision block are not written. */
   int64_t lse_out_batch_stride, lse_out_head_stride;
+  const int32_t* seq_start;        /* DEVICE [B] or NULL.  Packed (ragged) batches: sample b's rows start
+                                      seq_start[b] rows into hidden, q, k, lse and lse_out (added to
+                                      b * batch_stride, which a packed caller sets to 0), e.g. the cu_seqlens of a
+                                      batch stored back to back without padding.  With it, seq_rows must be the
+                                      total number of rows q and k hold. */
+  const int32_t* seq_start_out;    /* DEVICE [B] or NULL: the same for hidden_out.  Output lengths depend on the
+                                      data, so these are offsets the caller reserves (capacities), not lengths. */
 } lightkv_layer_args_t;
 
 #define LIGHTKV_MAX_TEXT_RANGES 8
@@ -301,6 +308,10 @@ typedef struct {
   int64_t src_page_stride, dst_page_stride;
   uint32_t* status;                /* DEVICE, may be NULL */
   void* stream;
+  const int32_t* src_seq_start;    /* DEVICE [B] or NULL: first token of sample b inside a packed source cache */
+  const int32_t* dst_seq_start;    /* ... (contiguous form: token offset added to b * batch_stride; paged form:
+                                      added to the token index before the block-table lookup); in place both
+                                      must be the same pointer */
 } lightkv_kv_args_t;
 
 int lightkv_compact_kv(const lightkv_plan_t* plan, const lightkv_kv_args_t* args);

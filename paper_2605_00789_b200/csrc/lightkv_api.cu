@@ -365,7 +365,8 @@ int lightkv_compact_kv(const lightkv_plan_t* p, const lightkv_kv_args_t* a) {
   if (in_place != (a->v_src == a->v_dst)) return LIGHTKV_ERR_INVALID_ARG;
   if (in_place && (a->src_batch_stride != a->dst_batch_stride || a->src_head_stride != a->dst_head_stride ||
                    a->src_row_stride != a->dst_row_stride || a->src_page_stride != a->dst_page_stride ||
-                   (a->page_size > 0 && a->src_block_table != a->dst_block_table)))
+                   (a->page_size > 0 && a->src_block_table != a->dst_block_table) ||
+                   a->src_seq_start != a->dst_seq_start))
     return LIGHTKV_ERR_INVALID_ARG;
   const void* ptrs[4] = {a->k_src, a->v_src, a->k_dst, a->v_dst};
   for (const void* q : ptrs) if (!aligned16(q)) return LIGHTKV_ERR_INVALID_ARG;

@@ -205,8 +205,8 @@ __device__ inline void load4<__nv_bfloat16>(const __nv_bfloat16* p, float (&f)[4
 
 template <typename T>
 __global__ void __launch_bounds__(256)
-fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_stride, int vis_begin,
-               int d, int metric, Workspace ws) {
+fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_stride, const int* __restrict__ seq_start,
+               int vis_begin, int d, int metric, Workspace ws) {
   grid_dependency_sync();
   __shared__ float As[FD_TA][FD_KC + 1];
   __shared__ float Bs[FD_TB][FD_KC + 1];
@@ -225,7 +225,7 @@ fd_simt_kernel(const T* __restrict__ hidden, int64_t batch_stride, int64_t row_s
   const int e0 = blockIdx.x * FD_TA;
   if (e0 >= n_a) return;
   const int ne = min(FD_TA, n_a - e0);
-  const T* x = hidden + size_t(b) * batch_stride + size_t(vis_begin) * row_stride;
+  const T* x = hidden + size_t(b) * batch_stride + size_t((seq_start ? seq_start[b] : 0) + vis_begin) * row_stride;
 
   if (tid < FD_TA) {
     if (tid < ne) {
@@ -319,9 +319,10 @@ cudaError_t launch_fd_simt(const LayerLaunch& L) {
   if (L.dtype == LIGHTKV_BF16)
     return launch_kernel(fd_simt_kernel<__nv_bfloat16>, grid, 256, 0, L.stream, 1,
                          static_cast<const __nv_bfloat16*>(L.a->hidden), L.a->hidden_batch_stride,
-                         L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.divergence, L.ws);
+                         L.a->hidden_row_stride, L.a->seq_start, L.a->vis_begin, L.hidden, L.divergence, L.ws);
   return launch_kernel(fd_simt_kernel<float>, grid, 256, 0, L.stream, 1, static_cast<const float*>(L.a->hidden),
-                       L.a->hidden_batch_stride, L.a->hidden_row_stride, L.a->vis_begin, L.hidden, L.divergence, L.ws);
+                       L.a->hidden_batch_stride, L.a->hidden_row_stride, L.a->seq_start, L.a->vis_begin, L.hidden,
+                       L.divergence, L.ws);
 }
 
 // =====================================================================================================
@@ -340,6 +341,7 @@ struct XiSimtArgs {
   const float* lse; int64_t lse_bs, lse_hs;        // caller's row log-sum-exp (ATTN_LSE) or nullptr
   float* lse_out; int64_t lse_out_bs, lse_out_hs;  // receives the row log-sum-exp (ATTN_FULL) or nullptr
   const int* n_vis;
+  const int* seq_start;                            // first row of each sample in q, k, lse, lse_out (packed batches) or nullptr
   int vis_begin, n_text_after, bidirectional;
   int n_q_heads, n_kv_heads, dh;
   TextSet text;
@@ -360,8 +362,9 @@ xi_simt_kernel(XiSimtArgs<T> a, Workspace ws) {
   if (t0 >= n) return;
   const int nq = min(XI_TQ, n - t0);
   const int hk = h / (a.n_q_heads / a.n_kv_heads);
-  const T* qh = a.q + size_t(b) * a.q_bs + size_t(h) * a.q_hs;
-  const T* kh = a.k + size_t(b) * a.k_bs + size_t(hk) * a.k_hs;
+  const int row0 = a.seq_start ? a.seq_start[b] : 0;
+  const T* qh = a.q + size_t(b) * a.q_bs + size_t(h) * a.q_hs + size_t(row0) * a.q_rs;
+  const T* kh = a.k + size_t(b) * a.k_bs + size_t(hk) * a.k_hs + size_t(row0) * a.k_rs;
   const float scale2 = 1.4426950408889634f / sqrtf((float)dh);      // logits in log2 units
   const int vis_begin = a.vis_begin;
   const int n_seq = vis_begin + n + a.n_text_after;                   // keys of this sample
@@ -428,7 +431,7 @@ xi_simt_kernel(XiSimtArgs<T> a, Workspace ws) {
         v[c] = ok[c] ? Ss[r * (XI_TK + 1) + lane + 32 * c] : -INFINITY;
       }
       if (a.lse) {
-        const float l2 = a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_i] * 1.4426950408889634f;
+        const float l2 = a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + row0 + s_i] * 1.4426950408889634f;
         float p = (txt[0] ? exp2f(v[0] - l2) : 0.f) + (txt[1] ? exp2f(v[1] - l2) : 0.f);
         for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
         l_txt[i] += p;
@@ -456,7 +459,7 @@ xi_simt_kernel(XiSimtArgs<T> a, Workspace ws) {
       if (r < nq) {
         ws.xi_h[(size_t(b) * a.n_q_heads + h) * ws.cap_in + t0 + r] = a.lse ? l_txt[i] : l_txt[i] / l_all[i];
         if (a.lse_out)
-          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + vis_begin + t0 + r] =
+          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + row0 + vis_begin + t0 + r] =
               (m_run[i] + log2f(l_all[i])) * 0.6931471805599453f;
       }
     }
@@ -475,7 +478,8 @@ static cudaError_t launch_xi_simt_t(const LayerLaunch& L) {
   x.lse = L.xi_mode == LIGHTKV_XI_ATTN_LSE ? a->lse : nullptr; x.lse_bs = a->lse_batch_stride; x.lse_hs = a->lse_head_stride;
   x.lse_out = L.xi_mode == LIGHTKV_XI_ATTN_FULL ? a->lse_out : nullptr;
   x.lse_out_bs = a->lse_out_batch_stride; x.lse_out_hs = a->lse_out_head_stride;
-  x.n_vis = a->n_vis; x.vis_begin = a->vis_begin; x.n_text_after = a->n_text_after; x.bidirectional = a->bidirectional;
+  x.n_vis = a->n_vis; x.seq_start = a->seq_start;
+  x.vis_begin = a->vis_begin; x.n_text_after = a->n_text_after; x.bidirectional = a->bidirectional;
   x.n_q_heads = L.n_q_heads; x.n_kv_heads = L.n_kv_heads; x.dh = dh; x.text = L.text;
   const cudaError_t e = ensure_dynamic_smem(xi_simt_kernel<T>, 160 * 1024);
   if (e != cudaSuccess) return e;
@@ -753,15 +757,16 @@ merge_rows_kernel(const T* __restrict__ src, int64_t src_bs, int64_t src_rs,
                   int d, int vis_begin, int n_text_after, int cap_in, int cap_out,
                   const int* __restrict__ n_vis, const int* __restrict__ n_vis_out,
                   const int* __restrict__ grp_off, const int* __restrict__ grp_src,
-                  const float* __restrict__ weight) {
+                  const float* __restrict__ weight, const int* __restrict__ seq_start,
+                  const int* __restrict__ seq_start_out) {
   grid_dependency_sync();
   constexpr int V = Vec<T>::n;
   const int b = blockIdx.y, row = blockIdx.x;
   const int n_in = n_vis ? min(n_vis[b], cap_in) : cap_in;
   const int n_out = n_vis_out[b];
   if (row >= vis_begin + n_out + n_text_after) return;
-  const T* sb = src + size_t(b) * src_bs;
-  T* orow = out + size_t(b) * out_bs + size_t(row) * out_rs;
+  const T* sb = src + size_t(b) * src_bs + size_t(seq_start ? seq_start[b] : 0) * src_rs;
+  T* orow = out + size_t(b) * out_bs + size_t((seq_start_out ? seq_start_out[b] : 0) + row) * out_rs;
   const int chunks = d / V;
   if (row < vis_begin || row >= vis_begin + n_out) {
     const T* srow = sb + size_t(row < vis_begin ? row : row - n_out + n_in) * src_rs;
@@ -831,12 +836,12 @@ cudaError_t launch_merge_rows(const LayerLaunch& L) {
         static_cast<const __nv_bfloat16*>(a->hidden), a->hidden_batch_stride, a->hidden_row_stride,
         static_cast<__nv_bfloat16*>(a->hidden_out), a->hidden_out_batch_stride, a->hidden_out_row_stride,
         L.hidden, a->vis_begin, a->n_text_after, L.ws.cap_in, L.ws.cap_out, a->n_vis, a->n_vis_out,
-        a->grp_off, a->grp_src, a->weight);
+        a->grp_off, a->grp_src, a->weight, a->seq_start, a->seq_start_out);
   return launch_kernel(merge_rows_kernel<float>, grid, 256, 0, L.stream, 1,
         static_cast<const float*>(a->hidden), a->hidden_batch_stride, a->hidden_row_stride,
         static_cast<float*>(a->hidden_out), a->hidden_out_batch_stride, a->hidden_out_row_stride,
         L.hidden, a->vis_begin, a->n_text_after, L.ws.cap_in, L.ws.cap_out, a->n_vis, a->n_vis_out,
-        a->grp_off, a->grp_src, a->weight);
+        a->grp_off, a->grp_src, a->weight, a->seq_start, a->seq_start_out);
 }
 
 // =====================================================================================================
@@ -851,7 +856,9 @@ struct KvAddr {
   int64_t batch_stride, head_stride, row_stride, page_stride;
   const int* table;       // nullptr = contiguous
   int page_size, max_blocks;
+  const int* seq_start;   // first token of each sample (packed caches) or nullptr
   __device__ inline int64_t token(int b, int n) const {
+    if (seq_start) n += seq_start[b];
     if (!table) return int64_t(b) * batch_stride + int64_t(n) * row_stride;
     const int page = table[size_t(b) * max_blocks + n / page_size];
     return int64_t(page) * page_stride + int64_t(n % page_size) * row_stride;
@@ -1031,9 +1038,9 @@ kv_move_kernel(T* __restrict__ k_buf, T* __restrict__ v_buf, KvAddr ad, int n_kv
 cudaError_t launch_kv_compact(const KvLaunch& K) {
   const lightkv_kv_args_t* a = K.a;
   KvAddr sa{a->src_batch_stride, a->src_head_stride, a->src_row_stride, a->src_page_stride,
-            a->page_size > 0 ? a->src_block_table : nullptr, a->page_size, a->max_blocks};
+            a->page_size > 0 ? a->src_block_table : nullptr, a->page_size, a->max_blocks, a->src_seq_start};
   KvAddr da{a->dst_batch_stride, a->dst_head_stride, a->dst_row_stride, a->dst_page_stride,
-            a->page_size > 0 ? a->dst_block_table : nullptr, a->page_size, a->max_blocks};
+            a->page_size > 0 ? a->dst_block_table : nullptr, a->page_size, a->max_blocks, a->dst_seq_start};
   const int ch_host = K.head_dim * (K.dtype == LIGHTKV_BF16 ? 2 : 4) / 16;
   if (2 * K.n_kv_heads * ch_host >= 65536) return cudaErrorInvalidValue;      // range of the unit decode
   const unsigned magic_ch = (unsigned)(((1ull << 32) + ch_host - 1) / ch_host);

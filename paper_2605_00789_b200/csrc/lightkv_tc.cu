@@ -102,6 +102,7 @@ struct XiSched {
 
 struct XiTcArgs {
   const int* n_vis;
+  const int* seq_start;              // first row of each sample in q, k, lse, lse_out (packed batches) or nullptr
   float* xi_h;
   uint32_t* status;
   const float* lse;                  // [B, H, N] row log-sum-exp (natural log) from the caller, or nullptr
@@ -168,7 +169,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   // log-sum-exp, only the tiles that hold prompt keys (J lies before the vision block, so it is visible)
   const int kt_lo = LSE ? a.text.begin / BK : 0;
   const int nkt_lse = a.text.end > a.text.begin ? (a.text.end - 1) / BK + 1 - kt_lo : 0;
-  struct Item { int h, b, t0, nq, s_first, nkt, n_seq, nsub; };   // nsub: halves of 64 keys the item visits
+  struct Item { int h, b, t0, nq, s_first, nkt, n_seq, nsub, row0, bc; };   // nsub: halves of 64 keys the item visits;
+                                                                           // row0, bc: row offset and batch coordinate of the TMA loads
   // item -> (query tile, head, sample).  The (sample, head) pairs are taken in groups of XT_HEAD_GROUP whose keys
   // stay in L2 together; inside a group the list runs over the query tiles from the longest rows to the shortest,
   // all pairs of the group for each, so that the work left for the last tickets is short.
@@ -186,6 +188,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     it.n_seq = a.vis_begin + n + a.n_text_after;
     it.nsub = LSE ? 2 * nkt_lse : ((a.bidirectional ? it.n_seq : it.s_first + it.nq) - 1) / XT_SUB + 1;
     it.nkt = (it.nsub + 1) / 2;
+    it.row0 = a.seq_start ? a.seq_start[it.b] : 0;        // packed batch: one long row axis, batch coordinate 0
+    it.bc = a.seq_start ? 0 : it.b;
     return true;
   };
 
@@ -228,7 +232,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         if (nq_loaded > 0 && !mbar_wait(q_empty, (nq_loaded - 1) & 1, abort_flag)) break;
         mbar_expect_tx(q_full, TILE_BYTES);
 #pragma unroll
-        for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.s_first, it.h, it.b);
+        for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.row0 + it.s_first, it.h, it.bc);
         ++nq_loaded;
         const int hk = it.h / a.group;
         bool ok = true;
@@ -238,7 +242,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
           mbar_expect_tx(&k_full[s], KT_BYTES);
 #pragma unroll
           for (int hf = 0; hf < HALVES; ++hf)
-            tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, (kt_lo + kt) * BK, hk, it.b);
+            tma_load_4d(k_s + s * KT_BYTES + hf * KHALF_BYTES, &k_map, &k_full[s], hf * 64, it.row0 + (kt_lo + kt) * BK, hk, it.bc);
         }
         if (!ok) break;
       }
@@ -327,7 +331,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
           }
 
           if (LSE) {                                      // normaliser known: only the prompt columns count
-            const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + s_first + r] * 1.4426950408889634f : 0.f;
+            const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + it.row0 + s_first + r] * 1.4426950408889634f : 0.f;
             const unsigned int tm = (unsigned int)a.text.mask64(j0);
             float st = 0.f;
 #pragma unroll
@@ -439,7 +443,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       if (r < nq && !*abort_flag) {
         a.xi_h[(size_t(b) * a.n_q_heads + h) * a.cap_in + it.t0 + r] = LSE ? l_txt : l_txt / l_all;
         if (!LSE && a.lse_out)
-          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + s_first + r] =
+          a.lse_out[size_t(b) * a.lse_out_bs + size_t(h) * a.lse_out_hs + it.row0 + s_first + r] =
               fmaf(m_run, sc, log2f(l_all)) * 0.6931471805599453f;
       }
     }
@@ -461,13 +465,14 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   const lightkv_layer_args_t* a = L.a;
   const int rows = a->seq_rows > 0 ? a->seq_rows : a->vis_begin + L.ws.cap_in + a->n_text_after;
   CUtensorMap qm, km;
-  if (!make_map_bhnd(&qm, a->q, L.head_dim, rows, L.n_q_heads, L.batch, a->q_row_stride, a->q_head_stride,
+  const int map_batch = a->seq_start ? 1 : L.batch;       // packed batch: every sample lives on one row axis
+  if (!make_map_bhnd(&qm, a->q, L.head_dim, rows, L.n_q_heads, map_batch, a->q_row_stride, a->q_head_stride,
                      a->q_batch_stride, 128) ||
-      !make_map_bhnd(&km, a->k, L.head_dim, rows, L.n_kv_heads, L.batch, a->k_row_stride, a->k_head_stride,
+      !make_map_bhnd(&km, a->k, L.head_dim, rows, L.n_kv_heads, map_batch, a->k_row_stride, a->k_head_stride,
                      a->k_batch_stride, XT_KEY_TILE))
     return cudaErrorInvalidValue;
   XiTcArgs x;
-  x.n_vis = a->n_vis; x.xi_h = L.ws.xi_h; x.status = a->status; x.cap_in = L.ws.cap_in;
+  x.n_vis = a->n_vis; x.seq_start = a->seq_start; x.xi_h = L.ws.xi_h; x.status = a->status; x.cap_in = L.ws.cap_in;
   x.lse = L.xi_mode == LIGHTKV_XI_ATTN_LSE ? a->lse : nullptr; x.lse_bs = a->lse_batch_stride; x.lse_hs = a->lse_head_stride;
   x.lse_out = L.xi_mode == LIGHTKV_XI_ATTN_FULL ? a->lse_out : nullptr;
   x.lse_out_bs = a->lse_out_batch_stride; x.lse_out_hs = a->lse_out_head_stride;
@@ -525,6 +530,7 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
 // ======================================================================================================
 struct FdTcArgs {
   const __nv_bfloat16* x;              // first vision row of sample 0
+  const int* seq_start;                // first row of each sample (packed batches) or nullptr
   int64_t batch_stride, row_stride;    // elements
   int d, batch;
   int metric;                          // LIGHTKV_FD_*
@@ -671,7 +677,8 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
   if (warp < 8) {
     // ---- gather: thread = 16-byte piece c of row slots g, g + 32, g + 64, g + 96 of every fill
     const int c = tid & 7, g = tid >> 3;
-    const unsigned char* xb = reinterpret_cast<const unsigned char*>(a.x + size_t(b) * a.batch_stride) + size_t(c_lo) * 128;
+    const unsigned char* xb = reinterpret_cast<const unsigned char*>(
+        a.x + size_t(b) * a.batch_stride + size_t(a.seq_start ? a.seq_start[b] : 0) * a.row_stride) + size_t(c_lo) * 128;
     const int* a_tok = a.ws.a_tok + size_t(b) * a.ws.cap_a;
     const int* b_tok = a.ws.b_tok + size_t(b) * a.ws.cap_b;
     // source row of slot t on even / odd fills (they differ only when passes = 4), validity bits, and the
@@ -922,6 +929,7 @@ cudaError_t launch_fd_tc(const LayerLaunch& L) {
   const lightkv_layer_args_t* a = L.a;
   FdTcArgs f;
   f.x = static_cast<const __nv_bfloat16*>(a->hidden) + size_t(a->vis_begin) * a->hidden_row_stride;
+  f.seq_start = a->seq_start;
   f.batch_stride = a->hidden_batch_stride; f.row_stride = a->hidden_row_stride; f.d = L.hidden; f.batch = L.batch;
   f.metric = L.divergence; f.ws = L.ws; f.status = a->status;
   // Persistent CTAs, two per SM, no more than the plan expects tiles.  When that estimate leaves SMs idle,

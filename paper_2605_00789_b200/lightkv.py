@@ -67,7 +67,8 @@ class _LayerArgs(C.Structure):
                 ("map_event", C.c_void_p), ("fork_event", C.c_void_p), ("join_event", C.c_void_p),
                 ("n_text_ranges", C.c_int32), ("bidirectional", C.c_int32),
                 ("text_ranges", C.POINTER(C.c_int32)),
-                ("lse_out", C.c_void_p), ("lse_out_batch_stride", C.c_int64), ("lse_out_head_stride", C.c_int64)]
+                ("lse_out", C.c_void_p), ("lse_out_batch_stride", C.c_int64), ("lse_out_head_stride", C.c_int64),
+                ("seq_start", C.c_void_p), ("seq_start_out", C.c_void_p)]
 
 
 MAX_TEXT_RANGES = 8
@@ -86,7 +87,8 @@ class _KvArgs(C.Structure):
                 ("page_size", C.c_int32), ("max_blocks", C.c_int32),
                 ("src_block_table", C.c_void_p), ("dst_block_table", C.c_void_p),
                 ("src_page_stride", C.c_int64), ("dst_page_stride", C.c_int64),
-                ("status", C.c_void_p), ("stream", C.c_void_p)]
+                ("status", C.c_void_p), ("stream", C.c_void_p),
+                ("src_seq_start", C.c_void_p), ("dst_seq_start", C.c_void_p)]
 
 
 EXPORTS = ("lightkv_plan", "lightkv_plan_stage_info", "lightkv_plan_destroy", "lightkv_plan_retention",
@@ -227,13 +229,14 @@ def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin:
                 n_text_after: int = 0, text_begin: int = 0, text_end: Optional[int] = None,
                 q=None, k=None, lse=None, xi=None, n_vis=None, pos=None, stream=None,
                 trace_events=None, aux_stream=None, map_event=None, fork_event=None, join_event=None,
-                text_ranges=None, bidirectional: bool = False, lse_out=None) -> _LayerArgs:
+                text_ranges=None, bidirectional: bool = False, lse_out=None, seq_start=None, seq_start_out=None,
+                hidden_out=None) -> _LayerArgs:
     a = _LayerArgs()
     a.struct_size = C.sizeof(_LayerArgs)
     a.stage, a.vis_begin, a.n_text_after = stage, vis_begin, n_text_after
     a.text_begin, a.text_end = text_begin, vis_begin if text_end is None else text_end
     a.hidden, a.hidden_batch_stride, a.hidden_row_stride = hidden.data_ptr(), hidden.stride(0), hidden.stride(1)
-    ho = out.hidden_out
+    ho = out.hidden_out if hidden_out is None else hidden_out
     a.hidden_out, a.hidden_out_batch_stride, a.hidden_out_row_stride = ho.data_ptr(), ho.stride(0), ho.stride(1)
     if q is not None:
         a.seq_rows = q.shape[2]
@@ -265,6 +268,13 @@ def _layer_args(plan: Plan, stage: int, hidden, out: StageBuffers, *, vis_begin:
     a.bidirectional = int(bool(bidirectional))
     if lse_out is not None:
         a.lse_out, a.lse_out_batch_stride, a.lse_out_head_stride = lse_out.data_ptr(), lse_out.stride(0), lse_out.stride(1)
+    if seq_start is not None:
+        # packed batch: tensors of shape [1, rows, ...] hold the samples back to back; sample b starts at row
+        # seq_start[b], so the batch strides are 0 and q / k span all rows
+        a.seq_start, a.seq_start_out = seq_start.data_ptr(), _ptr(seq_start_out)
+        a.hidden_batch_stride = a.q_batch_stride = a.k_batch_stride = a.lse_batch_stride = a.lse_out_batch_stride = 0
+        if seq_start_out is not None:
+            a.hidden_out_batch_stride = 0
     if map_event is not None:         # a torch.cuda.Event that has been recorded once (torch creates it lazily)
         a.map_event = map_event.cuda_event
     if trace_events is not None:      # TRACE_EVENTS torch.cuda.Event objects (enable_timing=True), already created
@@ -277,7 +287,8 @@ def compress_layer(plan: Plan, stage: int, hidden, out: StageBuffers, **kw) -> N
     """lightkv_compress_layer.  hidden [B,N,d]; keywords: vis_begin, n_text_after, text_begin, text_end,
     q [B,H,N,dh], k [B,H_kv,N,dh] (any strides with a contiguous last dimension), lse [B,H,N] fp32,
     xi [B,cap_in] fp32, n_vis [B] int32, pos [B,cap_in] int32, stream, trace_events, aux_stream, map_event,
-    fork_event / join_event, text_ranges [(begin, end), ...], bidirectional, lse_out [B,H,N] fp32."""
+    fork_event / join_event, text_ranges [(begin, end), ...], bidirectional, lse_out [B,H,N] fp32,
+    seq_start / seq_start_out [B] int32 (packed batches), hidden_out (instead of out.hidden_out)."""
     a = _layer_args(plan, stage, hidden, out, **kw)
     _check(library().lightkv_compress_layer(plan.handle, C.byref(a)), "lightkv_compress_layer")
 
@@ -294,7 +305,8 @@ def compress_layer_builtin_ws(plan: Plan, stage: int, hidden, out: StageBuffers,
 
 def compact_kv(plan: Plan, stage: int, out: StageBuffers, k_src, v_src, k_dst, v_dst, *, vis_begin: int,
                n_text_after: int = 0, mode: int = KV_MERGE, n_vis=None, page_size: int = 0,
-               src_block_table=None, dst_block_table=None, stream=None) -> None:
+               src_block_table=None, dst_block_table=None, stream=None, src_seq_start=None,
+               dst_seq_start=None) -> None:
     """lightkv_compact_kv.  Contiguous: k/v [B,H_kv,N,dh] views (any batch/head/row strides).
     Paged: k/v page pools [n_pages, H_kv, page_size, dh] views and int32 block tables [B, max_blocks]."""
     a = _KvArgs()
@@ -315,4 +327,8 @@ def compact_kv(plan: Plan, stage: int, out: StageBuffers, k_src, v_src, k_dst, v
         a.dst_batch_stride, a.dst_head_stride, a.dst_row_stride = k_dst.stride(0), k_dst.stride(1), k_dst.stride(2)
     a.status = _ptr(out.status)
     a.stream = _stream_handle(stream)
+    if src_seq_start is not None:     # packed caches: sample b's first token; contiguous batch strides become 0
+        a.src_seq_start, a.src_batch_stride = src_seq_start.data_ptr(), 0
+    if dst_seq_start is not None:
+        a.dst_seq_start, a.dst_batch_stride = dst_seq_start.data_ptr(), 0
     _check(library().lightkv_compact_kv(plan.handle, C.byref(a)), "lightkv_compact_kv")

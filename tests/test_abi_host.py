@@ -39,8 +39,8 @@ def test_struct_layouts_match_the_header(L, tmp_path):
 int main(void) {
   printf("%zu %zu\\n", sizeof(lightkv_config_t), offsetof(lightkv_config_t, direction));
   printf("%zu %zu\\n", sizeof(lightkv_stage_info_t), offsetof(lightkv_stage_info_t, reserved));
-  printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, lse_out_head_stride));
-  printf("%zu %zu\\n", sizeof(lightkv_kv_args_t), offsetof(lightkv_kv_args_t, stream));
+  printf("%zu %zu\\n", sizeof(lightkv_layer_args_t), offsetof(lightkv_layer_args_t, seq_start_out));
+  printf("%zu %zu\\n", sizeof(lightkv_kv_args_t), offsetof(lightkv_kv_args_t, dst_seq_start));
   return 0;
 }
 ''')
@@ -50,8 +50,8 @@ int main(void) {
     k = L.lightkv
     got = [(C.sizeof(k._Config), k._Config.direction.offset),
            (C.sizeof(k._StageInfo), k._StageInfo.reserved.offset),
-           (C.sizeof(k._LayerArgs), k._LayerArgs.lse_out_head_stride.offset),
-           (C.sizeof(k._KvArgs), k._KvArgs.stream.offset)]
+           (C.sizeof(k._LayerArgs), k._LayerArgs.seq_start_out.offset),
+           (C.sizeof(k._KvArgs), k._KvArgs.dst_seq_start.offset)]
     assert got == rows
 
 

@@ -295,6 +295,66 @@ def test_in_place_equals_out_of_place_bit_for_bit():
     plan.close()
 
 
+# ---- packed (ragged) batches: samples back to back on one row axis ----------------------------------------------
+
+@pytest.mark.parametrize("engine,xi_mode,in_place", [("auto", "attn", False), ("simt", "attn", False),
+                                                     ("auto", "lse", False), ("auto", "attn", True)])
+def test_packed_batch_with_row_offsets(engine, xi_mode, in_place):
+    """Three samples of different lengths (one of them empty) stored without padding: every tensor has one row
+    axis and seq_start / seq_start_out say where a sample begins.  Same results as the padded form."""
+    import torch
+    import paper_2605_00789_b200 as L
+    wl = S.workload("small")
+    plan = H.make_plan(wl, xi_mode=xi_mode, engine=engine)
+    full = np.arange(wl.n_vis, dtype=np.int32)
+    rng = np.random.default_rng(6)
+    pos = [full, np.sort(rng.choice(full, 101, replace=False)).astype(np.int32), full[:0]]
+    inp = H.prepare_stage(wl, 0, pos)
+    info = plan.stage_info(0)
+    vb, bsz = inp["vis_begin"], 3
+    lens = [vb + int(n) for n in inp["n_vis"]]
+    start = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    start_out = (np.arange(bsz + 1) * (vb + info.cap_out)).astype(np.int32)
+    dev = "cuda"
+
+    def pack(a, axis):          # [B, (H,) N, w] -> [1, (H,) total, w]
+        return np.concatenate([np.take(a[b], range(lens[b]), axis - 1) for b in range(bsz)], axis - 1)[None]
+
+    hid = H.to_device(pack(inp["hidden"], 1), "bf16", dev)
+    q, k, v = (H.to_device(pack(inp[n], 2), "bf16", dev) for n in ("q", "k", "v"))
+    out = L.StageBuffers(plan, 0, vb + info.cap_out, dev)
+    hidden_out = torch.full((1, int(start_out[-1]), wl.hidden), float("nan"), dtype=torch.bfloat16, device=dev)
+    pos_pad = np.pad(inp["pos"], ((0, 0), (0, info.cap_in - inp["pos"].shape[1])), constant_values=-1)
+    kw = dict(vis_begin=vb, q=q, k=k, n_vis=torch.from_numpy(inp["n_vis"]).to(dev), pos=torch.from_numpy(pos_pad).to(dev),
+              seq_start=torch.from_numpy(start[:-1].copy()).to(dev), seq_start_out=torch.from_numpy(start_out[:-1].copy()).to(dev),
+              hidden_out=hidden_out)
+    if xi_mode == "lse":
+        lse = H.oracle_lse(inp, wl.n_q_heads, wl.n_kv_heads)                      # [B, H, N] padded
+        kw["lse"] = torch.from_numpy(pack(lse[:, :, :, None], 2)[..., 0].astype(np.float32)).to(dev)   # [1, H, total]
+    L.compress_layer(plan, 0, hid, out, **kw)
+    if in_place:
+        k_dst, v_dst, dst_start = k, v, kw["seq_start"]
+    else:
+        k_dst = torch.full((1, wl.n_kv_heads, int(start_out[-1]), wl.head_dim), float("nan"), dtype=torch.bfloat16, device=dev)
+        v_dst, dst_start = k_dst.clone(), kw["seq_start_out"]
+    L.compact_kv(plan, 0, out, k, v, k_dst, v_dst, vis_begin=vb, n_vis=kw["n_vis"], src_seq_start=kw["seq_start"],
+                 dst_seq_start=dst_start)
+    torch.cuda.synchronize()
+    gpu = {name: getattr(out, name).cpu().numpy() for name in
+           ("n_vis_out", "pos_out", "dst", "weight", "grp_off", "grp_src", "xi_out", "status")}
+    n_out = gpu["n_vis_out"]
+    ho = hidden_out.float().cpu().numpy()[0]
+    kd, vd = k_dst.float().cpu().numpy()[0], v_dst.float().cpu().numpy()[0]
+    so = start if in_place else start_out
+    gpu["hidden_out"] = np.stack([ho[start_out[b]:start_out[b] + vb + info.cap_out] for b in range(bsz)])
+    rows = vb + info.cap_out
+    gpu["k_out"] = np.stack([np.pad(kd[:, so[b]:so[b] + vb + n_out[b]], ((0, 0), (0, rows - vb - n_out[b]), (0, 0))) for b in range(bsz)])
+    gpu["v_out"] = np.stack([np.pad(vd[:, so[b]:so[b] + vb + n_out[b]], ((0, 0), (0, rows - vb - n_out[b]), (0, 0))) for b in range(bsz)])
+    ref = H.oracle_stage(wl, 0, inp, xi_mode)
+    H.compare_stage(wl, 0, inp, ref, gpu)
+    plan.close()
+
+
 # ---- the variants the paper ablates: Euclidean pair scores, reverse message direction ---------------------------
 
 @pytest.mark.parametrize("metric", ["l2sq", "l2"])
