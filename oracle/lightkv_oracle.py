@@ -194,6 +194,25 @@ def select_edges(fd: np.ndarray, r: int) -> np.ndarray:
     return m
 
 
+def select_edges_literal(fd: np.ndarray, n_window: int, keep: float) -> np.ndarray:
+    """Step 2 read to the letter (the alternative to select_edges): ALL |A| x |B|
+    pairs are ranked by ascending FD (ties: lower A index, then lower B index) and
+    the floor(rho * n / 2) lowest form T_rho, rho = 1 - keep, n = tokens of the
+    window.  One-to-one matching is not enforced in either direction: an A node
+    may get several edges, and the number of A nodes that disappear (those with
+    at least one edge) depends on the data -- which is why the counts the paper
+    prints (a fraction 1 - rho remains; 576 -> 288) cannot come from this rule.
+    Kept for comparison; the library implements select_edges."""
+    n_a, n_b = fd.shape
+    m = np.zeros((n_a, n_b), dtype=np.int64)
+    k = int(math.floor((1.0 - keep) * n_window / 2.0 + 1e-9))
+    if k <= 0 or n_b == 0:
+        return m
+    flat = np.argsort(fd, axis=None, kind="stable")[:min(k, n_a * n_b)]   # row-major: A index, then B index
+    m[np.unravel_index(flat, fd.shape)] = 1
+    return m
+
+
 # --------------------------------------------------------------------------
 # Step 3 (Eq. "message-passing"): xi-weighted aggregation into B
 # --------------------------------------------------------------------------
@@ -228,6 +247,38 @@ def message_passing(xa: np.ndarray, xb: np.ndarray, xi_a: np.ndarray, xi_b: np.n
 # --------------------------------------------------------------------------
 # One compression stage over the vision tokens of one sample (Steps 1-5)
 # --------------------------------------------------------------------------
+
+def compress_vision_literal(x: np.ndarray, pos: np.ndarray, xi: np.ndarray,
+                            tiles: Sequence[Tuple[int, int]], w: int, keep: float) -> Dict[str, np.ndarray]:
+    """One stage with the literal edge rule (select_edges_literal): an A node may
+    send its message to several B nodes, so the map is many-to-many and is
+    returned as the per-window adjacency instead of one slot per token.
+    Returns x_out / pos_out (survivors in ascending position) and, per window,
+    (ia, ib, M)."""
+    x = np.asarray(x, dtype=F64)
+    pos = np.asarray(pos, dtype=np.int64)
+    xi = np.asarray(xi, dtype=F64)
+    win = window_of(pos, tiles, w)
+    alive = np.ones(len(x), dtype=bool)
+    x_new = x.copy()
+    edges = []
+    for wid in np.unique(win):
+        members = np.nonzero(win == wid)[0]
+        members = members[np.argsort(pos[members], kind="stable")]
+        ia, ib = bipartition(members)
+        if len(ib) == 0:
+            continue
+        m = select_edges_literal(feature_divergence(x[ia], x[ib]), len(members), keep)
+        xb_new, _, _ = message_passing(x[ia], x[ib], xi[ia], xi[ib], m)
+        touched = m.sum(axis=0) > 0
+        x_new[ib[touched]] = xb_new[touched]
+        alive[ia[m.sum(axis=1) > 0]] = False
+        edges.append((ia, ib, m))
+    survivors = np.nonzero(alive)[0]
+    survivors = survivors[np.argsort(pos[survivors], kind="stable")]
+    return {"x_out": x_new[survivors], "pos_out": pos[survivors], "survivor": survivors,
+            "n_out": np.int64(len(survivors)), "edges": edges}
+
 
 def compress_vision(x: np.ndarray, pos: np.ndarray, xi: np.ndarray,
                     tiles: Sequence[Tuple[int, int]], w: int, keep: float,

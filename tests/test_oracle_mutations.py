@@ -183,6 +183,10 @@ def _compress_vision_ignores_the_direction(x, pos, xi, tiles, w, keep, metric="c
     return O_compress_vision(x, pos, xi, tiles, w, keep, metric, "a2b")
 
 
+def _select_edges_literal_counts_tokens_not_pairs(fd, n_window, keep):
+    return O_select_edges_literal(fd, n_window, 1.0 - 2.0 * (1.0 - keep)) if keep > 0.5 else O_select_edges_literal(fd, 2 * n_window, keep)
+
+
 def _window_of_swapped_axes(pos, tiles, w):
     return O_window_of(pos, [(c, r) for r, c in tiles], w)
 
@@ -200,6 +204,7 @@ O_attention_rows, O_message_passing, O_window_of = O.attention_rows, O.message_p
 O_retention, O_compact_kv = O.retention, O.compact_kv
 O_row_logsumexp, O_scaled_logits = O.row_logsumexp, O.scaled_logits
 O_divergence, O_compress_vision = O.divergence, O.compress_vision
+O_select_edges_literal = O.select_edges_literal
 
 MUTATIONS = [
     ("feature_divergence", _fd_wrong_sign),
@@ -223,6 +228,7 @@ MUTATIONS = [
     ("scaled_logits", _scaled_logits_always_causal),
     ("divergence", _divergence_l2sq_without_the_cross_term),
     ("compress_vision", _compress_vision_ignores_the_direction),
+    ("select_edges_literal", _select_edges_literal_counts_tokens_not_pairs),
     ("window_of", _window_of_swapped_axes),
     ("retention", _retention_counts_the_compression_layer_as_compressed),
     ("compact_kv", _compact_kv_ignores_the_weights),

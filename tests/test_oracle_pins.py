@@ -459,6 +459,37 @@ def test_selection_agrees_with_exhaustive_matching(n, keep):
     assert m.sum() == r and (m.sum(axis=1) <= 1).all()          # one edge per A node at most
 
 
+def test_literal_edge_rule_lets_one_a_node_feed_two_b_nodes():
+    """Step 2 to the letter: the floor(rho n / 2) lowest PAIRS, whatever nodes they join.  A hand case: A0 lies
+    between B0 and B1 and close to both, A1 is far from everything; with two pairs allowed both go to A0."""
+    xa = np.array([[1.0, 1.0, 0.0], [0.0, 0.0, 1.0]])           # A0, A1
+    xb = np.array([[1.0, 0.9, 0.0], [0.9, 1.0, 0.0]])           # B0, B1
+    fd = O.feature_divergence(xa, xb)
+    m = O.select_edges_literal(fd, 4, 0.0)                       # rho = 1: floor(4 / 2) = 2 pairs
+    np.testing.assert_array_equal(m, [[1, 1], [0, 0]])
+    np.testing.assert_array_equal(O.select_edges(fd, 2), [[1, 0], [1, 0]])    # the adopted rule: one edge per A node
+                                                                              # (ties go to the lower B index)
+    # the count of pairs is the printed floor(rho v / 2); the number of tokens that disappear is at most that
+    for n, keep in ((16, 0.5), (36, 0.5), (36, 0.7), (7, 0.5)):
+        rng = np.random.default_rng(n)
+        f = rng.uniform(0, 2, ((n + 1) // 2, n // 2))
+        mm = O.select_edges_literal(f, n, keep)
+        k = int(np.floor((1 - keep) * n / 2 + 1e-9))
+        assert mm.sum() == k and (mm.sum(axis=1) > 0).sum() <= k
+        assert f[mm == 1].max(initial=-1) <= f[mm == 0].min(initial=9)       # they are the lowest pairs
+    # through a whole stage: halving 576 tokens this way leaves MORE than 288 (at most 144 pairs per 576 tokens),
+    # which is why the library does not use this rule; A0's message reaches both B nodes with weight xi_A0
+    x, pos, xi, tiles, w, keep = _case(31, n=36)
+    res = O.compress_vision_literal(x, pos, xi, tiles, w, keep)
+    assert int(res["n_out"]) >= 36 - 9
+    ia, ib, m = res["edges"][0]
+    for bi in np.nonzero(m.sum(axis=0))[0]:
+        src = ia[m[:, bi] == 1]
+        want = (xi[ib[bi]] * x[ib[bi]] + (xi[src, None] * x[src]).sum(0)) / (xi[ib[bi]] + xi[src].sum())
+        o = int(np.nonzero(res["survivor"] == ib[bi])[0][0])
+        np.testing.assert_allclose(res["x_out"][o], want, rtol=1e-13)
+
+
 def test_many_a_nodes_may_share_one_b_node():
     x = np.array([[1, 0.01], [1, 0.0], [1, -0.01], [0, 1.0], [1, 0.02], [-1, 0.0]])
     res = O.compress_vision(x, np.arange(6), np.ones(6), [(1, 6)], 1, 0.5)
