@@ -49,24 +49,28 @@ static bool make_map_bhnd(CUtensorMap* map, const void* base, int width, int row
 // xi per head on tensor cores (Eq. "attention-factor" over the softmax rows of Eq. "attention-matrix").
 //
 // A work item is (tile of 128 vision queries, head, sample).  Persistent CTAs, two per SM, draw items from a
-// ticket counter in global memory (items of one head are neighbours in the list, so concurrent CTAs share
-// its K in L2; within a head the longest rows come first).  Warp 0 is the scheduler and the TMA producer: it
+// ticket counter in global memory (the list interleaves groups of 64 (sample, head) pairs whose K stays in L2
+// together, longest rows first inside a group).  Warp 0 is the scheduler and the TMA producer: it
 // publishes the ticket to the other roles through a two-slot ring in shared memory, streams the item's Q tile
 // once and its K tiles (128 keys) through a 2-stage ring; the next item's Q and first K tiles are requested as
 // soon as the MMAs of the current item have drained, i.e. while its last tiles are still in the softmax warps.
-// Warp 1 issues S = Q K^T (128 x 128 x dh, bf16 -> fp32) into one of two TMEM accumulators.  Warps 2-5 own one
-// query row per thread (= TMEM lane): they pull the accumulator into registers in two halves of 64 logits,
-// release it, and add exp(logit - reference) to two sums per row (all visible keys / prompt keys J).
+// Warp 1 issues S = Q K^T (128 x 128 x dh, bf16 -> fp32) into one of two TMEM accumulators.  Warps 2-9 are
+// the softmax warps, two threads per query row (= TMEM lane): a thread pulls 32 of the 64 logits of a half of the
+// accumulator into registers (the warp that takes the last piece releases the accumulator) and adds
+// exp(logit - reference) to two sums (all visible keys / prompt keys J); the two threads of a row combine their
+// references and sums once per item through shared memory.
 // Output per head: sum_J / sum_all.
 //
 // The kernel is bound by the exponentials (one per logit on the special-function unit, 16 per clock per SM,
 // against one MMA per tile), so the softmax arithmetic is kept to three instructions per logit:
-//   * the reference subtracted before the exponential is the row's maximum over the FIRST 64 keys only
+//   * the reference subtracted before the exponential is the thread's maximum over its FIRST 32 keys only
 //     (softmax is invariant to the reference; fp32 holds exp of any later logit up to 88 above it), so the
 //     other tiles need no maximum and no rescaling;
-//   * on halves that need neither the causal mask nor the prompt mask, every fourth exponential is evaluated
-//     on the FMA pipe instead (range reduction + cubic, relative error 7.5e-5), which takes a quarter of the
-//     load off the special-function unit.
+//   * on halves that need neither the causal mask nor the prompt mask, every eighth exponential is evaluated
+//     on the FMA pipe instead (range reduction + cubic, relative error 7.5e-5).  With the softmax warps alone
+//     on an SM a quarter is the best share; in the whole kernel, which runs into the power limit (SM clock
+//     about 1.78 GHz instead of 1.965), the dozen instructions of the cubic cost more than the special-function
+//     slot they free, and an eighth measured fastest (none: +1 %, a quarter: +4 %, three eighths: +10 %).
 // A row whose sum left the fp32 range (a later logit more than 88 above the first keys' maximum) is found at
 // the end of its item, which is then appended to a list in global memory; a second launch of the kernel
 // (SAFE) walks that list with a running maximum and rescaling on every half, as an ordinary online softmax
@@ -375,12 +379,12 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
           if (m_run == -INFINITY) continue;                // this thread has not seen a key yet
           const float ms = m_run * sc;
           if (!edge && !in_j) {
-            // the bulk: every fourth exponential on the FMA pipe
+            // the bulk: every eighth exponential on the FMA pipe
             float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const float x = fmaf(v[i], sc, -ms);
-              part[i & 3] += (i & 3) == 3 ? ex2_fma(x) : ex2(x);
+              part[i & 3] += (i & 7) == 7 ? ex2_fma(x) : ex2(x);
             }
             l_all += (part[0] + part[1]) + (part[2] + part[3]);
           } else {
