@@ -142,17 +142,20 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   constexpr uint32_t TILE_BYTES = HALVES * 16384;          // Q tile: 128 rows x DH bf16
   constexpr uint32_t KHALF_BYTES = BK * 128;               // BK key rows x 64 columns
   constexpr uint32_t KT_BYTES = HALVES * KHALF_BYTES;      // K tile: BK rows x DH bf16
+  // With the caller's normaliser an item is one or two key tiles and the kernel is bound by reading Q from HBM:
+  // then the Q tile is double buffered (two items' Q in flight per CTA) and one K stage is enough.
+  constexpr int QBUF = LSE ? 2 : 1, KSTAGES = LSE ? 1 : XT_STAGES;
   const unsigned int n_items = SAFE ? a.sched->n_redo : unsigned(a.n_qt) * a.n_q_heads * a.batch;
   if (n_items == 0) return;                                // nothing on the list: the usual case of the second launch
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* q_s = base;
-  unsigned char* k_s = base + TILE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(base + TILE_BYTES + KT_BYTES * XT_STAGES);
-  uint64_t* q_full = bars;
-  uint64_t* q_empty = bars + 1;                // every MMA that reads the Q tile has completed
-  uint64_t* k_full = bars + 2;                 // [XT_STAGES]
+  unsigned char* q_s = base;                   // [QBUF] Q tiles
+  unsigned char* k_s = base + QBUF * TILE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + QBUF * TILE_BYTES + KT_BYTES * KSTAGES);
+  uint64_t* q_full = bars;                     // [2]
+  uint64_t* q_empty = bars + 2;                // [2] every MMA that reads the Q tile has completed
+  uint64_t* k_full = bars + 4;                 // [XT_STAGES]
   uint64_t* k_empty = k_full + XT_STAGES;      // [XT_STAGES]
   uint64_t* s_full = k_empty + XT_STAGES;      // [XT_SBUF]
   uint64_t* s_empty = s_full + XT_SBUF;        // [XT_SBUF]
@@ -198,8 +201,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   };
 
   if (threadIdx.x == 0) {
-    mbar_init(q_full, 1);
-    mbar_init(q_empty, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1); }
     for (int i = 0; i < XT_STAGES; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
     for (int i = 0; i < XT_SBUF; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 8); }
     for (int i = 0; i < 2; ++i) { mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 9); }
@@ -224,7 +226,10 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       for (;;) {
         const uint32_t slot = n & 1;
         if (!mbar_wait(&item_empty[slot], ((n >> 1) & 1) ^ 1, abort_flag)) break;
-        const unsigned int t = atomicAdd(SAFE ? &a.sched->safe_ticket : &a.sched->ticket, 1u);
+        // items of the LSE form are all alike: a fixed round-robin split balances them and saves the atomic's
+        // round trip, which would otherwise be a good part of such a short item
+        const unsigned int t = LSE ? blockIdx.x + n * gridDim.x
+                                   : atomicAdd(SAFE ? &a.sched->safe_ticket : &a.sched->ticket, 1u);
         const int item = t < n_items ? (SAFE ? a.redo_list[t] : int(t)) : -1;
         item_slot[slot] = item;
         mbar_arrive(&item_full[slot]);                 // release: the slot is written before the arrival is seen
@@ -232,17 +237,19 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         if (item < 0) break;
         Item it;
         if (!decode(item, it) || it.nkt == 0) continue;
-        // the Q tile is free once every MMA of the previous item has completed
-        if (nq_loaded > 0 && !mbar_wait(q_empty, (nq_loaded - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(q_full, TILE_BYTES);
+        // a Q buffer is free once every MMA of the item that used it last has completed
+        const uint32_t qb = nq_loaded % QBUF, q_use = nq_loaded / QBUF;
+        if (q_use > 0 && !mbar_wait(&q_empty[qb], (q_use - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(&q_full[qb], TILE_BYTES);
 #pragma unroll
-        for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(q_s + hf * 16384, &q_map, q_full, hf * 64, it.row0 + it.s_first, it.h, it.bc);
+        for (int hf = 0; hf < HALVES; ++hf)
+          tma_load_4d(q_s + qb * TILE_BYTES + hf * 16384, &q_map, &q_full[qb], hf * 64, it.row0 + it.s_first, it.h, it.bc);
         ++nq_loaded;
         const int hk = it.h / a.group;
         bool ok = true;
         for (int kt = 0; kt < it.nkt; ++kt, ++kf) {
-          const uint32_t s = kf % XT_STAGES;
-          if (!mbar_wait(&k_empty[s], ((kf / XT_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          const uint32_t s = kf % KSTAGES;
+          if (!mbar_wait(&k_empty[s], ((kf / KSTAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
           mbar_expect_tx(&k_full[s], KT_BYTES);
 #pragma unroll
           for (int hf = 0; hf < HALVES; ++hf)
@@ -273,24 +280,26 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
         if (item < 0) break;
         Item it;
         if (!decode(item, it) || it.nkt == 0) continue;
-        if (!mbar_wait(q_full, nq_used & 1, abort_flag)) break;
+        const uint32_t qb = nq_used % QBUF;
+        if (!mbar_wait(&q_full[qb], (nq_used / QBUF) & 1, abort_flag)) break;
+        const uint64_t q_off = uint64_t(qb * (TILE_BYTES >> 4));
         bool ok = true;
         for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
-          const uint32_t s = kc % XT_STAGES, buf = kc % XT_SBUF;
+          const uint32_t s = kc % KSTAGES, buf = kc % XT_SBUF;
           if (!mbar_wait(&s_empty[buf], ((kc / XT_SBUF) & 1) ^ 1, abort_flag) ||
-              !mbar_wait(&k_full[s], (kc / XT_STAGES) & 1, abort_flag)) { ok = false; break; }
+              !mbar_wait(&k_full[s], (kc / KSTAGES) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint64_t stage_off = uint64_t(s * (KT_BYTES >> 4));     // the address field counts 16-byte units
           const uint32_t d_addr = tmem_base + buf * BK;
           // the last tile of an odd number of halves needs its first 64 keys only
           const uint32_t idesc = (2 * kt + 2 > it.nsub) ? idesc_half : idesc_full;
 #pragma unroll
-          for (int kk = 0; kk < DH / 16; ++kk) umma_bf16(d_addr, q_desc[kk], k_desc[kk] + stage_off, idesc, kk > 0);
+          for (int kk = 0; kk < DH / 16; ++kk) umma_bf16(d_addr, q_desc[kk] + q_off, k_desc[kk] + stage_off, idesc, kk > 0);
           umma_commit(&k_empty[s]);
           umma_commit(&s_full[buf]);
         }
         if (!ok) break;
-        umma_commit(q_empty);
+        umma_commit(&q_empty[qb]);
         ++nq_used;
       }
     }
@@ -317,6 +326,9 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
       if (!decode(item, it)) continue;
       const int h = it.h, b = it.b, nq = it.nq, s_first = it.s_first;
       float m_run = -INFINITY, l_all = 0.f, l_txt = 0.f;
+      // the caller's normaliser of this row, in log2 units (fetched before the first wait: its latency hides there)
+      float l2 = 0.f;
+      if (LSE && r < nq) l2 = a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + it.row0 + s_first + r] * 1.4426950408889634f;
       for (int kt = 0; kt < it.nkt; ++kt, ++kc) {
         const uint32_t buf = kc % XT_SBUF;
         const bool landed = mbar_wait(&s_full[buf], (kc / XT_SBUF) & 1, abort_flag);
@@ -335,7 +347,6 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
           }
 
           if (LSE) {                                      // normaliser known: only the prompt columns count
-            const float l2 = r < nq ? a.lse[size_t(b) * a.lse_bs + size_t(h) * a.lse_hs + it.row0 + s_first + r] * 1.4426950408889634f : 0.f;
             const unsigned int tm = (unsigned int)a.text.mask64(j0);
             float st = 0.f;
 #pragma unroll
@@ -491,7 +502,9 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   // As many CTAs as stay resident (two per SM) draw work items from a ticket counter; with the caller's
   // log-sum-exp an item is one or two key tiles, otherwise up to the whole row.
   const dim3 grid((unsigned)std::min<long long>(n_items, XT_CTAS * sm_count()));
-  const size_t smem = size_t(L.head_dim / 64) * (16384 + size_t(XT_STAGES) * XT_KEY_TILE * 128) + 1024 + 256 + 1536;
+  // Q tiles + K ring (LSE: two Q tiles, one K stage; otherwise one Q tile, XT_STAGES K stages) + barriers + exchange
+  const size_t smem = size_t(L.head_dim / 64) * (x.lse ? 2 * 16384 + XT_KEY_TILE * 128
+                                                        : 16384 + size_t(XT_STAGES) * XT_KEY_TILE * 128) + 1024 + 256 + 1536;
   cudaError_t e = cudaMemsetAsync(x.sched, 0, sizeof(XiSched), L.stream);      // tickets and list length start at 0
   if (e != cudaSuccess) return e;
   auto launch = [&](auto kernel, dim3 g) -> cudaError_t {
