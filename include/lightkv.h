@@ -24,8 +24,8 @@
  * attention mass vision token i puts on the prompt tokens, summed over heads
  * (Eq. "attention-factor").  Merged A nodes are dropped (Step 4) and the
  * survivors are emitted in their original order (Step 5).  The same map is
- * applied to the layer's K/V cache ("key and value tokens are compressed
- * simultaneously", appendix "Method overview").
+ * applied to the layer's K/V cache, which the method shrinks together with the
+ * tokens (appendix "Method overview").
  */
 #ifndef LIGHTKV_H_
 #define LIGHTKV_H_
@@ -80,8 +80,8 @@ extern "C" {
 #define LIGHTKV_FD_L2SQ   1      /* squared Euclidean distance            */
 #define LIGHTKV_FD_L2     2      /* Euclidean distance                    */
 
-/* direction of the messages (paragraph "Token message passing": "the reverse direction can be defined
- * analogously") */
+/* direction of the messages (paragraph "Token message passing" leaves the reverse direction open as the
+ * analogue of the forward one) */
 #define LIGHTKV_DIR_A2B 0        /* A nodes (1st, 3rd, ... token of a window) are merged into B nodes: the method */
 #define LIGHTKV_DIR_B2A 1        /* the sets swap roles: B nodes are merged into their best A node; a window of
                                     n tokens can then lose at most floor(n / 2) of them                           */

@@ -286,8 +286,8 @@ def compress_vision(x: np.ndarray, pos: np.ndarray, xi: np.ndarray,
     """x [n, d], pos [n] (original flat positions, any storage order), xi [n].
 
     metric: pair score of Step 2 (see divergence).  direction: "a2b" passes messages
-    from X_A to X_B as the method does; "b2a" is the reverse direction that paragraph
-    "Token message passing" says can be defined analogously: the two sets swap
+    from X_A to X_B as the method does; "b2a" is the reverse direction, which paragraph
+    "Token message passing" leaves as the analogue of the forward one: the two sets swap
     roles, so B nodes are merged into their best A node and at most |B| = floor(n / 2)
     tokens of a window disappear.
 
@@ -360,7 +360,7 @@ def compress_sequence(hidden: np.ndarray, vis_begin: int, n_vis: int, pos: np.nd
 
 
 # --------------------------------------------------------------------------
-# K/V reduction ("key and value tokens are compressed simultaneously")
+# K/V reduction (the cache shrinks together with the tokens: appendix "Method overview")
 # --------------------------------------------------------------------------
 
 def compact_kv(kv: np.ndarray, vis_begin: int, n_vis: int, dst: np.ndarray, weight: np.ndarray,

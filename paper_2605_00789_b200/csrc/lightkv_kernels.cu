@@ -845,7 +845,7 @@ cudaError_t launch_merge_rows(const LayerLaunch& L) {
 }
 
 // =====================================================================================================
-// K/V merge-compaction ("key and value tokens are compressed simultaneously for later layers").
+// K/V merge-compaction (the cache of a layer shrinks together with its tokens: appendix "Method overview").
 // The stage's merge map is applied per KV head; contiguous (strided) or paged (block-table) addressing
 // on either side.  One CTA per output token, five CTAs per SM; every thread resolves the token's group
 // itself (uniform, cached loads) and works on two 16-byte units and two group members at a time, i.e.
