@@ -264,8 +264,9 @@ int lightkv_compress_layer(const lightkv_plan_t* plan, const lightkv_layer_args_
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  *     that device current) and remembers it; make that first call outside any stream capture.
  *     LIGHTKV_ERR_CUDA if the lookup fails.
- *   - All calls on one device share the array, and it keeps what the previous call left.  Nothing
- *     in it has to start at zero (every kernel of the stage writes what the later ones read), but
+ *   - All calls on one device share the array, and it keeps what the previous call left.  The only
+ *     words that have to start at zero (the ticket counters of the xi kernel) are cleared by a 16-byte
+ *     cudaMemsetAsync on the stream inside every call; everything else is written before it is read.  But
  *     two calls whose kernels overlap on the GPU (different streams, no ordering between them)
  *     race on it: order such calls, or give all but one of them lightkv_compress_layer with their
  *     own workspace. */
