@@ -618,7 +618,9 @@ def main():
             cpu["one_thread"] = {"unavailable": str(exc)}
 
     if rank == 0:
-        launches_per_step = n_stages * 6
+        # per stage: window build, xi (+ its second launch for rows that left the fp32 range; none with a given
+        # log-sum-exp), FD, selection, hidden merge, K/V compaction (+ the move kernel when in place)
+        launches_per_step = n_stages * (6 + (1 if args.xi_mode == "full" else 0) + (1 if args.kv_in_place else 0))
         line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
