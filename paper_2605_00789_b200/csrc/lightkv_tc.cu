@@ -720,6 +720,15 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     const uint32_t slot0 = uint32_t(g) * 128 + (uint32_t(c ^ (g & 7)) << 4);   // swizzled offset of slot g; slot g+32t is 4096 t further
     const int chunk_shift = passes == 4 ? 1 : 0, chunk_mul = passes == 1 ? 2 : 1;
     float acc_e[4] = {0.f, 0.f, 0.f, 0.f}, acc_o[4] = {0.f, 0.f, 0.f, 0.f};
+    // columns of this thread's A row in the epilogue (row = TMEM lane): the B entries of the row's own window.
+    // Fetched here, two dependent loads deep, so that their latency hides behind the rows that stream below.
+    const int q = warp & 3, half = warp >> 2, row = q * 32 + lane, e = a0 + row;
+    int lo = 0x7fffffff, hi = 0;
+    if (e < a1) {
+      const int w = a.ws.a_win[size_t(b) * a.ws.cap_a + e];
+      lo = max(win_off[w] - a_off[w], b0) - b0;
+      hi = min(win_off[w + 1] - a_off[w + 1], b1) - b0;
+    }
 
     // rows the tile does not have and chunks past the hidden size are not fetched at all; the pieces of
     // the last chunk that lie past the hidden size are zero-filled
@@ -809,13 +818,8 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
     ok = ok && mbar_wait(acc_full, n_items & 1, abort_flag);
     ok = __all_sync(0xffffffffu, ok);                     // the TMEM loads below are warp-wide
     tc_fence_after();
-    const int q = warp & 3, half = warp >> 2, row = q * 32 + lane, e = a0 + row;
-    int lo = 0, hi = 0;
-    if (e < a1) {
-      const int w = a.ws.a_win[size_t(b) * a.ws.cap_a + e];
-      lo = max(win_off[w] - a_off[w], b0) - b0;
-      hi = min(win_off[w + 1] - a_off[w + 1], b1) - b0;
-    }
+    // columns some row of this warp needs: blocks of eight outside that range are skipped as a whole
+    const int lo_w = __reduce_min_sync(0xffffffffu, lo), hi_w = __reduce_max_sync(0xffffffffu, hi);
     const float na = row < cap_rows ? a_nrm[row] : 0.f;
     float best = 3.0e38f;
     int best_c = -1;
@@ -838,15 +842,20 @@ __global__ void __launch_bounds__(FT_LOADERS + 32, 2) fd_tc_kernel(FdTcArgs a) {
       for (int j = 0; j < 2; ++j) {
         const int c0 = half * 64 + j * 32;
         if (c0 >= n_cols) break;                          // warp-uniform
+        if (c0 + 32 <= lo_w || c0 >= hi_w) continue;      // warp-uniform
         float v[32];
         tmem_ld32(tmem_base + (uint32_t(q * 32) << 16) + c0, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int col = c0 + i;
-          if (col >= lo && col < hi) {
-            const float fd = pair_score(a.metric, v[i], na, b_nrm[col]);
-            if (fd < best) { best = fd; best_c = col; }
+        for (int blk = 0; blk < 4; ++blk) {
+          if (c0 + blk * 8 + 8 <= lo_w || c0 + blk * 8 >= hi_w) continue;   // warp-uniform
+#pragma unroll
+          for (int i = blk * 8; i < blk * 8 + 8; ++i) {
+            const int col = c0 + i;
+            if (col >= lo && col < hi) {
+              const float fd = pair_score(a.metric, v[i], na, b_nrm[col]);
+              if (fd < best) { best = fd; best_c = col; }
+            }
           }
         }
       }
