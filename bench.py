@@ -500,6 +500,27 @@ def main():
     barrier()
     clocks = sampler.stop()
     ms_step_one_stream = max_over_ranks(k_begin.elapsed_time(k_end), world, device) / ksteps
+    # the same one-stream schedule without events between the launches, replayed from a graph: the difference
+    # to the pass above is what recording an event after every kernel costs (launch latencies are exposed)
+    ms_one_stream_graph = None
+    if args.graph:
+        try:
+            torch.cuda.synchronize()
+            g1 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g1):
+                run_step(L, plan, wl, stages)
+            g1.replay()
+            barrier()
+            c_begin, c_end = ev(), ev()
+            c_begin.record()
+            for _ in range(ksteps):
+                g1.replay()
+            c_end.record()
+            barrier()
+            ms_one_stream_graph = max_over_ranks(c_begin.elapsed_time(c_end), world, device) / ksteps
+        except Exception as exc:      # noqa: BLE001
+            print(f"bench: one-stream graph capture refused ({exc})", file=sys.stderr)
+            torch.cuda.synchronize()
 
     ktime = {k: 0.0 for k in KERNELS}       # ms per step, summed over stages
     kstage = [{k: 0.0 for k in KERNELS} for _ in range(n_stages)]
@@ -630,6 +651,10 @@ def main():
                              if side is not None else "one stream"),
                 "cuda_graph": step_graph is not None,
                 "ms_per_step_one_stream": ms_step_one_stream,
+                "ms_per_step_one_stream_graph": ms_one_stream_graph,
+                "per_kernel_note": ("kernels / us_by_stage / roofline come from the one-stream pass with an event after "
+                                    "every launch (ms_per_step_one_stream); ms_per_step_one_stream_graph is the same "
+                                    "schedule without those events"),
                 "roofline": roofline, "kernels": kernels,
                 "us_by_stage": [{k: round(1e3 * v, 1) for k, v in ks.items()} for ks in kstage], "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                 "gpu_launches": launches_per_step * args.steps,
