@@ -36,10 +36,10 @@ KERNELS = ("window_build", "xi", "fd_best_partner", "select_map", "merge_hidden"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures (profiles/),
 # of the stage-0 launch, keyed by (workload, kernel); null where no capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("cfg2", "xi"): 401.53e6,                # profiles/xi_tc_kernel_cfg2_stage0.txt
-    ("cfg2", "fd_best_partner"): 193.35e6,   # profiles/fd_tc_kernel_cfg2_stage0.txt
-    ("cfg2", "merge_hidden"): 263.63e6,      # profiles/merge_rows_kernel_cfg2_stage0.txt
-    ("cfg2", "kv_compact"): 563.96e6,        # profiles/kv_compact_kernel_cfg2_stage0.txt
+    ("cfg2", "xi"): 401.05e6,                # profiles/xi_tc_kernel_cfg2_stage0.txt
+    ("cfg2", "fd_best_partner"): 192.91e6,   # profiles/fd_tc_kernel_cfg2_stage0.txt
+    ("cfg2", "merge_hidden"): 264.93e6,      # profiles/merge_rows_kernel_cfg2_stage0.txt
+    ("cfg2", "kv_compact"): 563.41e6,        # profiles/kv_compact_kernel_cfg2_stage0.txt
 }
 
 
