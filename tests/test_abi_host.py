@@ -120,6 +120,62 @@ def test_ragged_input_plans_hold_for_any_subset_of_the_grid(L):
     assert all(r.workspace_bytes >= e.workspace_bytes for r, e in zip(ragged, exact))
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_ragged_capacities_bound_what_the_oracle_produces_on_random_subsets(L, seed):
+    """The capacities of a ragged_input plan must hold whatever subset of the grid a sample enters with: run the
+    oracle stage by stage on random subsets (both message directions) and compare its counts with the plan's."""
+    import numpy as np
+    from oracle import lightkv_oracle as O
+    rng = np.random.default_rng(400 + seed)
+    tiles = [(int(rng.integers(6, 15)), int(rng.integers(6, 15))) for _ in range(int(rng.integers(1, 3)))]
+    smallest = min(min(t) for t in tiles)
+    windows = sorted((int(rng.integers(1, min(6, smallest) + 1)) for _ in range(3)), reverse=True)
+    keep = [float(k) for k in rng.uniform(0.5, 0.95, size=3).round(2)]
+    direction = ["a2b", "b2a"][seed % 2]
+    plan = L.Plan(batch=1, hidden=64, n_q_heads=2, n_kv_heads=2, head_dim=16, n_layers=8, tiles=tiles,
+                  layers=[2, 4, 6], windows=windows, keep=keep, max_text=8, ragged_input=True,
+                  direction=L.DIR_A2B if direction == "a2b" else L.DIR_B2A)
+    n_grid = sum(r * c for r, c in tiles)
+    for trial in range(4):
+        n0 = int(rng.integers(max(2, n_grid // 3), n_grid + 1))
+        pos = np.sort(rng.choice(n_grid, n0, replace=False))
+        for st in range(3):
+            info = plan.stage_info(st)
+            assert len(pos) <= info.cap_in
+            win = O.window_of(pos, tiles, windows[st])
+            counts = np.bincount(win, minlength=info.n_windows)
+            src = (counts + 1) // 2 if direction == "a2b" else counts // 2
+            assert src.sum() <= info.cap_a and (counts - src).sum() <= info.cap_b, (st, src.sum(), info.cap_a, info.cap_b)
+            x = rng.standard_normal((len(pos), 8))
+            res = O.compress_vision(x, pos, np.ones(len(pos)), tiles, windows[st], keep[st], direction=direction)
+            assert int(res["n_out"]) <= info.cap_out, (st, int(res["n_out"]), info.cap_out)
+            pos = res["pos_out"]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_exact_plans_agree_with_the_oracle_on_full_grids(L, seed):
+    """Where the plan calls its counts exact (the host simulation of the schedule), the oracle on a full grid must
+    produce exactly those counts, stage after stage; elsewhere the capacities must still bound them."""
+    import numpy as np
+    from oracle import lightkv_oracle as O
+    rng = np.random.default_rng(500 + seed)
+    side = int(rng.choice([8, 12, 16, 24]))
+    tiles = [(side, side)] * int(rng.integers(1, 3))
+    windows = [[4, 2, 1], [2, 2, 1], [4, 4, 2], [3, 2, 1]][seed % 4]
+    keep = [0.5, 0.5, 0.5] if seed % 2 == 0 else [0.5, 0.75, 0.5]
+    plan = L.Plan(batch=1, hidden=64, n_q_heads=2, n_kv_heads=2, head_dim=16, n_layers=8, tiles=tiles,
+                  layers=[2, 4, 6], windows=windows, keep=keep, max_text=8)
+    pos = np.arange(sum(r * c for r, c in tiles))
+    for st in range(3):
+        info = plan.stage_info(st)
+        x = rng.standard_normal((len(pos), 8))
+        res = O.compress_vision(x, pos, np.ones(len(pos)), tiles, windows[st], keep[st])
+        assert len(pos) <= info.cap_in and int(res["n_out"]) <= info.cap_out
+        if info.counts_exact:
+            assert len(pos) == info.cap_in and int(res["n_out"]) == info.cap_out
+        pos = res["pos_out"]
+
+
 def test_prompt_ranges_and_stream_events_are_checked_on_the_host(L):
     p = _plan(L)
     lib = L.library()
