@@ -306,6 +306,23 @@ def oracle_sample_step(wl, full_schedule=True):
     return oracle_sample_run(wl, per_stage, range(wl.n_stages) if full_schedule else [wl.n_stages - 1])
 
 
+def c_oracle_sample(wl, unit, per_stage):
+    """The plain C oracle (oracle/lightkv_oracle.c: simple loops, double precision, one thread) on the last stage of
+    sample 0: xi, the compression stage and the K/V compaction.  Returns a cpu_baseline-style dict."""
+    from oracle import c_oracle as OC
+    st = wl.n_stages - 1
+    inp = per_stage[st]
+    nv, vb = int(inp["n_vis"][0]), inp["vis_begin"]
+    t0 = time.perf_counter()
+    xi = OC.xi(inp["q"][0][:, :vb + nv], inp["k"][0][:, :vb + nv], vb, nv, [(0, vb)])
+    r = OC.compress(inp["hidden"][0, vb:vb + nv], inp["pos"][0, :nv], xi, wl.tiles, wl.windows[st], wl.keep[st])
+    for name in ("k", "v"):
+        OC.compact(inp[name][0][:, vb:vb + nv], r["dst"], r["weight"], r["n_out"])
+    t = time.perf_counter() - t0
+    return {"value": nv / t, "unit": unit, "cores": 1, "kind": "oracle (plain C)",
+            "sample": f"sample 0 of {wl.batch}, last stage only ({nv} vision tokens, {t:.1f} s)"}
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -625,18 +642,24 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        t, tok = oracle_sample_step(wl, full_schedule=True)
+        per_stage = oracle_sample_inputs(wl)                 # generated once, outside every timed interval
+        t, tok = oracle_sample_run(wl, per_stage, range(n_stages))
         cpu = {"value": tok / t, "unit": unit, "cores": blas_threads(), "kind": "oracle",
                "sample": f"sample 0 of {wl.batch}, all {n_stages} stages ({tok} vision tokens, {t:.1f} s)"}
         # the same oracle held to one thread, on the last stage of sample 0 (the smallest; bounded CPU time)
         try:
             from threadpoolctl import threadpool_limits
             with threadpool_limits(limits=1):
-                t1, tok1 = oracle_sample_step(wl, full_schedule=False)
+                t1, tok1 = oracle_sample_run(wl, per_stage, [n_stages - 1])
             cpu["one_thread"] = {"value": tok1 / t1, "unit": unit, "cores": 1,
                                  "sample": f"sample 0 of {wl.batch}, last stage only ({tok1} vision tokens, {t1:.1f} s)"}
         except Exception as exc:      # noqa: BLE001
             cpu["one_thread"] = {"unavailable": str(exc)}
+        # the plain C oracle (one thread by construction) on the same last stage of sample 0
+        try:
+            cpu["c_oracle_one_thread"] = c_oracle_sample(wl, unit, per_stage)
+        except Exception as exc:      # noqa: BLE001
+            cpu["c_oracle_one_thread"] = {"unavailable": str(exc)}
 
     if rank == 0:
         # per stage: window build, xi (+ its second launch for rows that left the fp32 range; none with a given

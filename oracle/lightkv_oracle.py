@@ -16,6 +16,8 @@ merge, permutation equivariance, keep = 1 identity, duplicated-token-first,
 and an exhaustive brute-force matching on <= 16 tokens.
 Parity unpinned by the paper (only self-consistency pins): window membership
 after the first stage, multi-tile grids, output order, and the K/V operator.
+A second oracle in plain C (lightkv_oracle.c), written separately, is compared
+with this one in tests/test_oracle_c.py.
 """
 from __future__ import annotations
 
