@@ -299,13 +299,6 @@ def oracle_sample_run(wl, per_stage, stage_list):
     return t_total, tokens
 
 
-def oracle_sample_step(wl, full_schedule=True):
-    """The CPU oracle on a bounded sample of the workload: sample 0 through the schedule (or its last
-    stage only).  Returns (seconds, vision tokens entering the stages it ran)."""
-    per_stage = oracle_sample_inputs(wl)
-    return oracle_sample_run(wl, per_stage, range(wl.n_stages) if full_schedule else [wl.n_stages - 1])
-
-
 def c_oracle_sample(wl, unit, per_stage):
     """The plain C oracle (oracle/lightkv_oracle.c: simple loops, double precision, one thread) on the last stage of
     sample 0: xi, the compression stage and the K/V compaction.  Returns a cpu_baseline-style dict."""
