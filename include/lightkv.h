@@ -140,9 +140,12 @@ typedef struct {
   int32_t reserved;
 } lightkv_stage_info_t;
 
-/* Build a plan.  HOST only, no CUDA call.  *out receives the plan.
- * Errors: INVALID_ARG (NULL, non-positive sizes, keep outside [0.5,1], w larger than a tile side,
- * layers not ascending), UNSUPPORTED (more windows per sample or more tiles than the kernels take). */
+/* Build a plan (Sec. "Hierarchical structure": the schedule Lambda, W, P; Eq. "complexity" for the accounting).
+ * HOST only, no CUDA call.  *out receives the plan, which the caller releases with lightkv_plan_destroy.
+ * Errors: INVALID_ARG (NULL, wrong struct_size, non-positive sizes, keep outside [0.5,1], w larger than a tile
+ * side, layers not ascending, an unknown dtype / xi_mode / engine / divergence / direction / ragged_input),
+ * UNSUPPORTED (more windows per sample or more tiles than the kernels take, more than 2^24 vision tokens, or a
+ * window that could hold more than 65535 tokens). */
 int  lightkv_plan(const lightkv_config_t* config, lightkv_plan_t** out);
 int  lightkv_plan_stage_info(const lightkv_plan_t* plan, int32_t stage, lightkv_stage_info_t* info);
 void lightkv_plan_destroy(lightkv_plan_t* plan);
@@ -246,9 +249,12 @@ typedef struct {
 
 #define LIGHTKV_TRACE_EVENTS 6
 
-/* Enqueue window build, xi, FD + best partner, selection + merge map and the
- * weighted merge of the hidden states.  Errors: INVALID_ARG, WORKSPACE (too
- * small), UNSUPPORTED (mode / dtype / engine combination), CUDA (launch failed). */
+/* Enqueue window build, xi, FD + best partner, selection + merge map and the weighted merge of the hidden states
+ * (Steps 1-5 of Sec. "LightKV"; Eq. "attention-factor", "similarity", "message-passing").  Nothing is allocated or
+ * synchronised; besides the kernels a 16-byte cudaMemsetAsync on `stream` clears the xi kernel's scheduler words
+ * in the workspace.  Errors: INVALID_ARG (NULL or misaligned buffers, strides below the row width, a prompt set
+ * outside [0, vis_begin], aux_stream without its two events, lse_out outside ATTN_FULL, ...), WORKSPACE (too small
+ * or not 256-byte aligned), CUDA (a launch failed).  Conditions only the device sees set bits of *status. */
 int lightkv_compress_layer(const lightkv_plan_t* plan, const lightkv_layer_args_t* args);
 
 /* The paper has no counterpart of this entry point; it exists for deployment only.
