@@ -128,6 +128,7 @@ constexpr int XT_CTAS = 2;           // CTAs per SM
 constexpr int XT_KEY_TILE = 128;     // keys per K tile and per MMA (the softmax warps read it as two halves of 64)
 constexpr int XT_SUB = 64;           // keys per half
 constexpr int XT_THREADS = 320;      // TMA / scheduler warp, MMA warp, eight softmax warps
+constexpr int XT_SAMPLE_CACHE = 256;  // samples whose token count and row offset are kept in shared memory
 constexpr int XT_HEAD_GROUP = 64;    // (sample, head) pairs whose work items are interleaved (their K: 64 x ~1 MB)
 
 // LSE: the caller supplied the row log-sum-exp (a.lse != nullptr).  SAFE: second launch, items from the list.
@@ -170,6 +171,10 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
   float* pair_m = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(bars) + 256);   // [128] each
   float* pair_all = pair_m + 128;
   float* pair_txt = pair_all + 128;
+  // per-sample token counts and row offsets, read once (every role decodes every item; a trip to global memory
+  // per item would be a good part of a short item); samples beyond the cache are read from global memory
+  int* s_nvis = reinterpret_cast<int*>(pair_txt + 128);    // [XT_SAMPLE_CACHE]
+  int* s_row0 = s_nvis + XT_SAMPLE_CACHE;                   // [XT_SAMPLE_CACHE]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // key tiles to visit: all tiles up to the last query's own key, or, when the caller supplies the row
@@ -187,7 +192,7 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     const int gsize = min(XT_HEAD_GROUP, n_hb - grp * XT_HEAD_GROUP);
     const int hb = grp * XT_HEAD_GROUP + within % gsize, qt = a.n_qt - 1 - within / gsize;
     it.h = hb % a.n_q_heads; it.b = hb / a.n_q_heads;
-    const int n = a.n_vis ? min(a.n_vis[it.b], a.cap_in) : a.cap_in;
+    const int n = it.b < XT_SAMPLE_CACHE ? s_nvis[it.b] : (a.n_vis ? min(a.n_vis[it.b], a.cap_in) : a.cap_in);
     it.t0 = qt * 128;
     if (it.t0 >= n) return false;
     it.nq = min(128, n - it.t0);
@@ -195,7 +200,8 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     it.n_seq = a.vis_begin + n + a.n_text_after;
     it.nsub = LSE ? 2 * nkt_lse : ((a.bidirectional ? it.n_seq : it.s_first + it.nq) - 1) / XT_SUB + 1;
     it.nkt = (it.nsub + 1) / 2;
-    it.row0 = a.seq_start ? a.seq_start[it.b] : 0;        // packed batch: one long row axis, batch coordinate 0
+    it.row0 = it.b < XT_SAMPLE_CACHE ? s_row0[it.b] : (a.seq_start ? a.seq_start[it.b] : 0);   // packed batch: one long
+                                                                                              // row axis, batch coordinate 0
     it.bc = a.seq_start ? 0 : it.b;
     return true;
   };
@@ -212,6 +218,10 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
     fence_barrier_init();
   }
   if (warp == 1) { tmem_alloc(tmem_slot, XT_SBUF * BK); tmem_relinquish(); }
+  for (int i = threadIdx.x; i < min(a.batch, XT_SAMPLE_CACHE); i += blockDim.x) {
+    s_nvis[i] = a.n_vis ? min(a.n_vis[i], a.cap_in) : a.cap_in;
+    s_row0[i] = a.seq_start ? a.seq_start[i] : 0;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -348,12 +358,19 @@ xi_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ 
 
           if (LSE) {                                      // normaliser known: only the prompt columns count
             const unsigned int tm = (unsigned int)a.text.mask64(j0);
-            float st = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if ((tm >> i) & 1u) st += ex2(fmaf(v[i], sc, -l2));
-            l_txt += st;
             l_all = 1.f;
+            if (tm == 0xffffffffu) {                      // all 32 keys are prompt keys: no tests, four chains
+              float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+              for (int i = 0; i < 32; ++i) part[i & 3] += ex2(fmaf(v[i], sc, -l2));
+              l_txt += (part[0] + part[1]) + (part[2] + part[3]);
+            } else if (tm != 0u) {
+              float st = 0.f;
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if ((tm >> i) & 1u) st += ex2(fmaf(v[i], sc, -l2));
+              l_txt += st;
+            }
             continue;
           }
           const bool in_j = j0 < a.text.end && j0 + 32 > a.text.begin;     // the columns reach into the prompt set J
@@ -504,7 +521,7 @@ cudaError_t launch_xi_tc(const LayerLaunch& L) {
   const dim3 grid((unsigned)std::min<long long>(n_items, XT_CTAS * sm_count()));
   // Q tiles + K ring (LSE: two Q tiles, one K stage; otherwise one Q tile, XT_STAGES K stages) + barriers + exchange
   const size_t smem = size_t(L.head_dim / 64) * (x.lse ? 2 * 16384 + XT_KEY_TILE * 128
-                                                        : 16384 + size_t(XT_STAGES) * XT_KEY_TILE * 128) + 1024 + 256 + 1536;
+                                                        : 16384 + size_t(XT_STAGES) * XT_KEY_TILE * 128) + 1024 + 256 + 1536 + 2 * XT_SAMPLE_CACHE * sizeof(int);
   cudaError_t e = cudaMemsetAsync(x.sched, 0, sizeof(XiSched), L.stream);      // tickets and list length start at 0
   if (e != cudaSuccess) return e;
   auto launch = [&](auto kernel, dim3 g) -> cudaError_t {
